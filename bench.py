@@ -1,0 +1,436 @@
+#!/usr/bin/env python
+"""Benchmark of one cross-layer MoE step (route -> schedule -> permute -> grouped expert FFN ->
+combine) on seeded synthetic inputs shaped like the benchmark configurations.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
+
+Prints ONE JSON line.  `value` is tokens of the chosen micro-batches per second with all inputs
+resident in HBM; `e2e` is the same through eb_step_host with pinned host buffers (host<->device
+copies inside the timed region).  With N > 1 (torchrun) every rank runs an independent replica
+on its own seeded batch (no collective on the data path); rank 0 reports the aggregate.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_07964_b200 import synth  # noqa: E402
+
+METRIC = "cross-layer MoE step tokens/s"
+UNIT = "tokens/s"
+KERNELS_PER_STEP = 13  # route 2, schedule 1, permute 5, expert FFN 4, combine 1
+
+# DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum), keyed by workload; see profiles/.  None until a capture exists.
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=d["hbm_gbs"], tensor=d["bf16_tflops"], tensor_sustained=d["bf16_tflops_sustained"], src="measured")
+    return dict(hbm=6650.0, tensor=1590.0, tensor_sustained=1400.0, src="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ts, line in self.lines:
+            f = [v.strip() for v in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                clk, mxc = float(f[0]), float(f[1])
+            except ValueError:
+                continue
+            mx = mxc
+            if t0 - 0.05 <= ts <= t1 + 0.15:
+                sm.append(clk)
+                for n, v in zip(names, f[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+        if not sm:
+            sm = [float(l.split(",")[0]) for _, l in self.lines[-3:] if l and l.split(",")[0].strip().replace(".", "").isdigit()]
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=mx, reasons=sorted(reasons), samples=len(sm))
+
+
+def timed(fn, reps: int):
+    """CUDA-event time of `reps` back-to-back calls on the current stream, in ms."""
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record()
+    for _ in range(reps):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b)
+
+
+def make_inputs(wl, device):
+    logits = synth.packed_logits(wl, device=device)
+    x = synth.packed_hidden(wl, device=device)
+    return logits, x
+
+
+def algorithmic_bytes(wl, group_off, n_groups):
+    sizes = np.diff(group_off[:n_groups + 1])
+    active = int((sizes > 0).sum())
+    R = int(sizes.sum())
+    w = wl.H * wl.I * 2
+    return dict(active_groups=active, rows=R,
+                gateup=active * 2 * w + R * wl.H * 2 + R * wl.I * 2,
+                down=active * w + R * wl.I * 2 + R * wl.H * 2,
+                gateup_flops=4.0 * wl.H * wl.I * R, down_flops=2.0 * wl.H * wl.I * R)
+
+
+# ----------------------------------------------------------------------------------------------
+def oracle_step_sample(wl, logits, x, weights_bf16_cpu, budget_s: float):
+    """The oracle's whole step on the CPU; the expert pass covers the first groups that fit the
+    time budget and the other stages are scaled to the same share of rows."""
+    from oracle import eb_oracle as O
+    dev = wl.expert_to_device()
+    t = {}
+    t0 = time.perf_counter()
+    idx, w, mb_load, mb_cnt = O.route(logits, wl.K, dev, wl.D, wl.tok_off, bool(wl.renorm_topk))
+    t["route"] = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    sched = O.schedule(mb_load, (1 << wl.N) - 1, wl.m, O.POLICY_MAXUTIL)
+    t["schedule"] = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    goff, gw, row_src, pos, xp, groups = O.permute(x, idx, sched["run_mask"], wl.layers, wl.tok_off, dev,
+                                                   wl.E, wl.K, wl.S, wl.D)
+    t["permute"] = time.perf_counter() - t0
+    R = int(goff[-1])
+    get = lambda wi: tuple(a.float().numpy() for a in weights_bf16_cpu(wi))
+    y = np.zeros((R, wl.H), dtype=np.float32)
+    t0 = time.perf_counter()
+    rows_done = 0
+    groups_done = 0
+    for g in range(len(gw)):
+        r0, r1 = int(goff[g]), int(goff[g + 1])
+        if r1 > r0:
+            wg, wu, wd = get(int(gw[g]))
+            y[r0:r1] = O.swiglu_mlp(xp[r0:r1], wg, wu, wd)
+            rows_done = r1
+            groups_done += 1
+        if time.perf_counter() - t0 > budget_s:
+            break
+    t["ffn"] = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    O.combine(y, pos, w, wl.K, wl.S)
+    t["combine"] = time.perf_counter() - t0
+    share = rows_done / max(R, 1)
+    tokens_run = sum(wl.T for j in range(wl.N) if (sched["run_mask"] >> j) & 1)
+    total = t["ffn"] + share * (t["route"] + t["schedule"] + t["permute"] + t["combine"])
+    return dict(tokens=tokens_run * share, seconds=total, share=share, groups=groups_done, rows=rows_done,
+                rows_total=R, stages=t)
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info()]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+def lazy_cpu_weights(wl, device):
+    """Callable giving one expert's (gate, up, down) as CPU bf16 tensors, generated on demand."""
+    cache = {}
+
+    def get(wi):
+        if wi not in cache:
+            l, e = divmod(wi, wl.E + wl.S)
+            cache[wi] = tuple(synth.expert_weight(wl, k, l, e, device).cpu() for k in ("gate", "up", "down"))
+        return cache[wi]
+    return get
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    gen_dev = "cuda" if torch.cuda.is_available() else "cpu"
+    logits, x = make_inputs(wl, gen_dev)
+    logits = logits.cpu().numpy()
+    x = x.float().cpu().numpy()
+    get = lazy_cpu_weights(wl, gen_dev)
+    budget = max(1.0, min(10.0, 150.0 / max(1, args.steps + args.warmup)))
+    # stage the weights of the groups the sample will touch outside the timed region
+    r = oracle_step_sample(wl, logits, x, get, budget)
+    for _ in range(max(0, args.warmup - 1)):
+        r = oracle_step_sample(wl, logits, x, get, budget)
+    tok = sec = 0.0
+    for _ in range(args.steps):
+        r = oracle_step_sample(wl, logits, x, get, budget)
+        tok += r["tokens"]
+        sec += r["seconds"]
+    value = tok / sec if sec > 0 else 0.0
+    sample = (f"oracle whole step on {wl.name}; expert pass over the first {r['groups']} non-empty groups "
+              f"({r['rows']} of {r['rows_total']} rows) within {budget:.0f} s, other stages scaled to that share")
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
+                ms_per_step=1000.0 * sec / max(1, args.steps), higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="f32", data="synthetic", impl="reference",
+                config=workload_config(wl),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=cpu_threads(), kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+def workload_config(wl):
+    return dict(workload=f"{wl.name}: L={wl.L} E={wl.E} K={wl.K} S={wl.S} H={wl.H} I={wl.I} D={wl.D} "
+                         f"map={wl.mapping} N={wl.N}x{wl.T} tokens at layers {wl.layers} m={wl.m} zipf_s={wl.zipf_s}",
+                policy="MaxUtil", seed=wl.seed,
+                l2="inputs larger than L2: each step streams the touched expert weights (GBs) from HBM")
+
+
+# ----------------------------------------------------------------------------------------------
+def run_ours(args, wl):
+    from paper_2608_07964_b200 import binding as B
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    device = f"cuda:{local}"
+    if rank:  # independent replicas: every rank draws its own batch and routing
+        wl = synth.Workload(**{**wl.__dict__, "seed": wl.seed + rank})
+    peaks = measured_peaks()
+
+    step = B.from_workload(wl, device=device)
+    wg, wu, wd = (synth.all_weights(wl, k, device) for k in ("gate", "up", "down"))
+    step.bind_weights(wg, wu, wd)
+    logits, x = make_inputs(wl, device)
+    T = wl.T_tot
+    step.logits[:T].copy_(logits)
+    step.x[:T].copy_(x)
+    batch = B.Batch(wl.tok_off, wl.layers)
+    m = wl.m
+    run = lambda: step.eb_step(batch, m)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing
+    for _ in range(args.warmup):
+        run()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    t0 = time.time()
+    ms = timed(run, args.steps)
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    barrier()
+    status = step.device_status()
+    sched = step.sched_result()
+    tokens_run = sum(wl.T for j in range(wl.N) if (sched["run_mask"] >> j) & 1)
+
+    # ---- per-kernel durations (events inside the library around every launch), same steps again
+    step.set_timing(True)
+    per = {}
+    for _ in range(args.steps):
+        run()
+        for k, v in step.kernel_ms().items():
+            per.setdefault(k, []).append(v)
+    step.set_timing(False)
+    kern_ms = {k: sum(v) / len(v) for k, v in per.items()}
+
+    # ---- end to end with host buffers
+    h_logits = logits.cpu().pin_memory()
+    h_x = x.cpu().pin_memory()
+    h_out = torch.empty((T, wl.H), dtype=torch.bfloat16).pin_memory()
+    run_host = lambda: step.eb_step_host(batch, m, h_logits, h_x, h_out)
+    for _ in range(min(args.warmup, 3)):
+        run_host()
+    barrier()
+    ms_e2e = timed(run_host, args.steps)
+    barrier()
+
+    # ---- reductions over ranks
+    tok_total, ms_max, ms_e2e_max = float(tokens_run), ms, ms_e2e
+    if dist is not None:
+        v = torch.tensor([ms, ms_e2e], device=device, dtype=torch.float64)
+        dist.all_reduce(v, op=dist.ReduceOp.MAX)
+        ms_max, ms_e2e_max = v.tolist()
+        tk = torch.tensor([tok_total], device=device, dtype=torch.float64)
+        dist.all_reduce(tk, op=dist.ReduceOp.SUM)
+        tok_total = tk.item()
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    meta = step.meta()
+    goff = step.group_off.cpu().numpy()
+    alg = algorithmic_bytes(wl, goff, meta["groups"])
+    ms_step = ms_max / args.steps
+    value = tok_total / (ms_step / 1e3)
+    # dominant kernel: the gate/up pass of the grouped expert FFN
+    t_gu = kern_ms.get("ffn_gateup", float("nan")) / 1e3
+    t_dn = kern_ms.get("ffn_down", float("nan")) / 1e3
+    hbm_time = alg["gateup"] / (peaks["hbm"] * 1e9)
+    tensor_time = alg["gateup_flops"] / (peaks["tensor"] * 1e12)
+    if hbm_time >= tensor_time:
+        achieved = alg["gateup"] / t_gu / 1e9
+        roof = dict(bound="hbm", achieved=achieved, peak=peaks["hbm"], unit="GB/s", frac=achieved / peaks["hbm"])
+    else:
+        achieved = alg["gateup_flops"] / t_gu / 1e12
+        roof = dict(bound="tensor", achieved=achieved, peak=peaks["tensor"], unit="TFLOP/s", frac=achieved / peaks["tensor"])
+    roof.update(kernel="ffn_gateup", peak_source=peaks["src"], traffic=NCU_TRAFFIC_BYTES.get(wl.name),
+                algorithmic_bytes=alg["gateup"], algorithmic_flops=alg["gateup_flops"], ms=t_gu * 1e3)
+    ffn_flops = alg["gateup_flops"] + alg["down_flops"]
+    ffn_bytes = alg["gateup"] + alg["down"]
+    t_ffn = t_gu + t_dn
+    move = 2 * (sum(wl.T for j in range(wl.N) if (sched["run_mask"] >> j) & 1) * wl.H + alg["rows"] * wl.H)
+    extra = dict(
+        kernel_ms=kern_ms,
+        ffn=dict(tflops=ffn_flops / t_ffn / 1e12, frac_tensor_peak=ffn_flops / t_ffn / 1e12 / peaks["tensor"],
+                 gbs=ffn_bytes / t_ffn / 1e9, frac_hbm=ffn_bytes / t_ffn / 1e9 / peaks["hbm"],
+                 down_gbs=alg["down"] / t_dn / 1e9, active_groups=alg["active_groups"], rows=alg["rows"]),
+        permute_gather_gbs=move / (kern_ms.get("permute_gather", float("nan")) / 1e3) / 1e9,
+        combine_gbs=move / (kern_ms.get("combine", float("nan")) / 1e3) / 1e9,
+    )
+    idle = idle_report(step, batch, wl, sched, B) if world == 1 and not args.no_idle else None
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        get = lazy_cpu_weights(wl, device)
+        lg, xx = logits.cpu().numpy(), x.float().cpu().numpy()
+        oracle_step_sample(wl, lg, xx, get, 4.0)          # stages the sampled weights on the host
+        r = oracle_step_sample(wl, lg, xx, get, 12.0)
+        cpu = dict(value=r["tokens"] / r["seconds"], unit=UNIT, cores=cpu_threads(), kind="oracle",
+                   sample=(f"oracle whole step; expert pass over the first {r['groups']} non-empty groups "
+                           f"({r['rows']} of {r['rows_total']} rows), other stages scaled to that share; "
+                           f"{r['seconds']:.1f} s of CPU work"))
+
+    h2d = T * wl.E * 4 + T * wl.H * 2
+    d2h = T * wl.H * 2 + 96
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+                data="synthetic", config=workload_config(wl), clocks=clocks,
+                e2e=dict(value=tok_total / (ms_e2e_max / args.steps / 1e3), unit=UNIT, h2d_bytes_per_step=h2d,
+                         d2h_bytes_per_step=d2h),
+                gpu_launches=KERNELS_PER_STEP * args.steps, roofline=roof, cpu_baseline=cpu,
+                tokens_per_step=tok_total, run_mask=sched["run_mask"], device_status=status, idle=idle, detail=extra)
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def idle_report(step, batch, wl, sched, B):
+    """Virtual-device idle fraction of the step, cross-layer versus each chosen micro-batch alone.
+
+    Token based: 1 - sum(W) / (D max(W)) from the routed loads.  Time based: the expert pass is run
+    on each virtual device's contiguous group range by itself (median of 5) and the same formula is
+    applied to the times; 'per layer' runs every chosen micro-batch's workload alone."""
+    D = wl.D
+    run = [j for j in range(wl.N) if (sched["run_mask"] >> j) & 1]
+    loads = step.mb_load[:wl.N].cpu().numpy().astype(np.int64)
+    joint = loads[run].sum(axis=0)
+    tok_cross = 1.0 - joint.sum() / (D * joint.max()) if joint.max() else 0.0
+    alone_cap = D * sum(int(loads[j].max()) for j in run)
+    tok_alone = 1.0 - joint.sum() / alone_cap if alone_cap else 0.0
+
+    def device_times():
+        out = []
+        for d in range(D):
+            f = lambda: step.eb_expert_ffn_grouped(device=d)
+            f()
+            out.append(statistics.median(timed(f, 1) for _ in range(5)))
+        return out
+
+    step.eb_step(batch, wl.m)
+    t_cross = device_times()
+    busy = cap = 0.0
+    for j in run:
+        one = B.Batch(wl.tok_off, wl.layers, 1 << j)
+        step.eb_schedule(one, 1, B.POLICY_ALL)
+        step.eb_permute(one)
+        tj = device_times()
+        busy += sum(tj)
+        cap += D * max(tj)
+    step.eb_step(batch, wl.m)
+    torch.cuda.synchronize()
+    return dict(token_cross_layer=tok_cross, token_per_layer=tok_alone,
+                time_cross_layer=1.0 - sum(t_cross) / (D * max(t_cross)),
+                time_per_layer=1.0 - busy / cap if cap else 0.0,
+                device_ms_cross_layer=t_cross, step_max_ms_cross_layer=max(t_cross), sum_max_ms_per_layer=cap / D)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c3init", "c4"])
+    ap.add_argument("--no-idle", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.workload == "c3init":
+        wl = synth.workload("c3", layers_override=tuple([0] * 16))
+        wl = synth.Workload(**{**wl.__dict__, "name": "c3init"})
+    else:
+        wl = synth.workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

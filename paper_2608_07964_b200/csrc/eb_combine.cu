@@ -1,0 +1,95 @@
+// eb_combine: weighted aggregation of Eq. 1 in gather form.
+//
+// One warp per token.  For every 16-byte column vector the warp loads the K + S expert-output
+// rows of the token (independent loads, all in flight together), accumulates in fp32 in the
+// fixed order k = 0..K-1 then s = 0..S-1, and stores bf16 (round to nearest even).  Gather form
+// means no atomics and a result that does not depend on scheduling.
+#include "eb_internal.cuh"
+
+namespace {
+
+constexpr int kWarps = 8;
+constexpr int kMaxSlots = EB_MAX_K + EB_MAX_S;
+
+__device__ __forceinline__ void fma8(float* acc, const uint4& v, float w) {
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 f = __bfloat1622float2(h[i]);
+    acc[2 * i] = fmaf(w, f.x, acc[2 * i]);
+    acc[2 * i + 1] = fmaf(w, f.y, acc[2 * i + 1]);
+  }
+}
+
+template <int KS>
+__global__ void __launch_bounds__(kWarps * 32)
+combine_kernel(int n_tok, int H, int K, const uint4* __restrict__ yp, const int32_t* __restrict__ pos,
+               const float* __restrict__ topk_w, uint4* __restrict__ out) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int t = blockIdx.x * kWarps + warp;
+  if (t >= n_tok) return;
+  int my_pos = lane < KS ? pos[(size_t)t * KS + lane] : -1;
+  float my_w = lane < K ? topk_w[(size_t)t * K + lane] : 1.0f;
+  if (__shfl_sync(0xffffffffu, my_pos, 0) < 0) return;  // micro-batch did not run: row untouched
+  const int vec = H / 8;
+  int p[KS];
+  float w[KS];
+#pragma unroll
+  for (int s = 0; s < KS; ++s) {
+    p[s] = __shfl_sync(0xffffffffu, my_pos, s);
+    w[s] = __shfl_sync(0xffffffffu, my_w, s);
+  }
+  for (int v = lane; v < vec; v += 32) {
+    uint4 r[KS];
+#pragma unroll
+    for (int s = 0; s < KS; ++s) r[s] = __ldg(yp + (size_t)p[s] * vec + v);
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int s = 0; s < KS; ++s) fma8(acc, r[s], w[s]);
+    uint4 o;
+    __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) oh[i] = __floats2bfloat162_rn(acc[2 * i], acc[2 * i + 1]);
+    out[(size_t)t * vec + v] = o;
+  }
+}
+
+typedef void (*combine_fn)(int, int, int, const uint4*, const int32_t*, const float*, uint4*);
+
+template <int KS>
+struct Table {
+  static void fill(combine_fn* f) {
+    f[KS] = combine_kernel<KS>;
+    Table<KS - 1>::fill(f);
+  }
+};
+template <>
+struct Table<0> {
+  static void fill(combine_fn*) {}
+};
+
+}  // namespace
+
+extern "C" eb_status eb_combine(eb_ctx* c, void* stream, const eb_batch* batch, const eb_sched_result* d_res,
+                                const void* yp, const int32_t* pos, const float* topk_w, void* out) {
+  if (!c) return EB_ERR_INVALID_ARG;
+  BatchParams bp;
+  eb_status s = ebi_make_batch(c, batch, &bp);
+  if (s != EB_OK) return s;
+  if (!d_res || !yp || !pos || !topk_w || !out) return ebi_fail(c, EB_ERR_INVALID_ARG, "null pointer");
+  if (!ebi_aligned16(yp) || !ebi_aligned16(out)) return ebi_fail(c, EB_ERR_INVALID_ARG, "yp / out must be 16-byte aligned");
+  if (bp.n_tok == 0) return EB_OK;
+  static combine_fn table[kMaxSlots + 1] = {};
+  static bool init = false;
+  if (!init) {
+    Table<kMaxSlots>::fill(table);
+    init = true;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  const int KS = c->cfg.K + c->cfg.S;
+  KernelTimer timer(c, EBK_COMBINE, st);
+  table[KS]<<<(bp.n_tok + kWarps - 1) / kWarps, kWarps * 32, 0, st>>>(bp.n_tok, c->cfg.H, c->cfg.K, (const uint4*)yp,
+                                                                     pos, topk_w, (uint4*)out);
+  EB_LAUNCH_CHECK(c, "combine");
+  return EB_OK;
+}

@@ -1,0 +1,516 @@
+// eb_expert_ffn_grouped: expert_i of Eq. 1 (bias-free SwiGLU MLP) for every (layer, expert) group
+// of a step in one grouped pass on the 5th-generation tensor cores.
+//
+// Two persistent launches over a device-built tile list (ragged groups, no padding rows in memory):
+//   gate/up : act[r, i] = silu(sum_h xp[r,h] Wg[i,h]) * (sum_h xp[r,h] Wu[i,h])      (bf16 out)
+//   down    : yp[r, h]  = sum_i act[r,i] Wd[h,i]                                      (bf16 out)
+// A tile is 128 rows x 256 accumulator columns.  For gate/up the 256 columns are 128 gate rows
+// and the matching 128 up rows of the weight matrices, loaded by two TMA copies into one
+// contiguous K-major operand, so one tcgen05.mma feeds both and the epilogue fuses SiLU * up.
+//
+// Per CTA (one per SM): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
+// warps 2..5 = epilogue (TMEM -> registers -> bf16 -> global).  Shared memory holds a 4-stage
+// ring of {A 128x64, B 256x64} bf16 tiles in the 128-byte swizzled K-major layout; TMEM holds two
+// 128x256 fp32 accumulators so the epilogue of tile i overlaps the MMAs of tile i+1.
+// Tiles of one group are ordered weight-tile-major, so CTAs working side by side share the
+// weight tile in L2 and every weight byte leaves HBM once per group.
+// Groups with at most 32 rows load a 32-row A box (the tensor core still multiplies 128 rows,
+// the extra rows are never stored), which keeps shared-memory fill traffic close to the weight
+// bytes in the weight-streaming regime.
+//
+// Every wait on an mbarrier is bounded: on expiry the kernel records EB_ERR_TIMEOUT in the
+// context status word, lets copies in flight land, frees its TMEM and returns.
+#include "eb_internal.cuh"
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int BN = 256;
+constexpr int kStages = 4;
+constexpr int kSmallRows = 32;
+constexpr int kABytes = BM * BK * 2;
+constexpr int kASmallBytes = kSmallRows * BK * 2;
+constexpr int kBBytes = BN * BK * 2;
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kThreads = 192;
+constexpr int kTmemCols = 512;
+constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr long long kSpinLimitCycles = 4000000000LL;
+
+// ---- PTX wrappers ----------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the limit expired or another thread of the CTA already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* s_abort, int* status) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t spin = 1;; ++spin) {
+    if (mbar_try(bar, parity)) return true;
+    if ((spin & 63u) == 0u) {
+      if (*s_abort) return false;
+      if (clock64() - t0 > kSpinLimitCycles) {
+        *s_abort = 1;
+        atomicExch(status, (int)EB_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 x bf16 -> fp32, M = 128, N = 256, K = 16
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// mbarrier arrives once all previously issued MMAs of this thread have completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory operand descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = 256, M = 128.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ float silu_mul(uint32_t g_bits, uint32_t u_bits) {
+  float g = __uint_as_float(g_bits), u = __uint_as_float(u_bits);
+  return g / (1.0f + __expf(-g)) * u;
+}
+
+// ---- the grouped GEMM kernel -----------------------------------------------------------------
+// PHASE 1: gate/up + SwiGLU (output tile 128 x 128);  PHASE 2: down (output tile 128 x 256).
+template <int PHASE>
+__global__ void __launch_bounds__(kThreads, 1)
+ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA_small,
+           const __grid_constant__ CUtensorMap tmB0, const __grid_constant__ CUtensorMap tmB1,
+           const int4* __restrict__ work, const int32_t* __restrict__ work_count, bf16* __restrict__ out,
+           int ld_out, int n_out, int k_total, int* status) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStages * kStageBytes);
+  // barrier indices: full[0..S), empty[S..2S), tmem_full[2S, 2S+2), tmem_empty[2S+2, 2S+4)
+  const uint32_t bar0 = base + kStages * kStageBytes;
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 + a); };
+  volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(bars + 2 * kStages + 4);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 2 * kStages + 5);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 4);
+    }
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    prefetch_tmap(&tmA);
+    prefetch_tmap(&tmA_small);
+    prefetch_tmap(&tmB0);
+    if (PHASE == 1) prefetch_tmap(&tmB1);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32((const void*)s_tmem), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+  const int n_work = work_count[PHASE - 1];
+  const int num_kb = (k_total + BK - 1) / BK;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int w = blockIdx.x; w < n_work; w += gridDim.x) {
+        const int4 it = __ldg(work + w);  // x = first row, y = valid rows, z = weight matrix, w = n tile
+        const bool small = it.y <= kSmallRows;
+        const uint32_t tx = (small ? kASmallBytes : kABytes) + kBBytes;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, s_abort, status)) goto done;
+          const uint32_t sa = base + stage * kStageBytes, sb = sa + kABytes;
+          mbar_expect_tx(full_bar(stage), tx);
+          tma_load_2d(sa, small ? &tmA_small : &tmA, kb * BK, it.x, full_bar(stage));
+          if (PHASE == 1) {
+            tma_load_3d(sb, &tmB0, kb * BK, it.w * 128, it.z, full_bar(stage));
+            tma_load_3d(sb + kBBytes / 2, &tmB1, kb * BK, it.w * 128, it.z, full_bar(stage));
+          } else {
+            tma_load_3d(sb, &tmB0, kb * BK, it.w * BN, it.z, full_bar(stage));
+          }
+          if (++stage == kStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int local = 0;
+      for (int w = blockIdx.x; w < n_work; w += gridDim.x, ++local) {
+        const int as = local & 1;
+        const uint32_t aphase = (local >> 1) & 1u;
+        if (!mbar_wait(tempty_bar(as), aphase ^ 1u, s_abort, status)) goto done;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + as * BN;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, s_abort, status)) goto done;
+          tc_fence_after();
+          const uint32_t sa = base + stage * kStageBytes, sb = sa + kABytes;
+          const uint64_t da = smem_desc(sa), db = smem_desc(sb);
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k)
+            umma_bf16(d_tmem, da + 2 * k, db + 2 * k, kIdesc, (kb | k) != 0 ? 1u : 0u);
+          umma_commit(empty_bar(stage));  // smem stage reusable once these MMAs have read it
+          if (++stage == kStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+        umma_commit(tfull_bar(as));  // accumulator complete
+      }
+    }
+  } else {
+    // ---------------- epilogue warps ----------------
+    const int q = warp & 3;  // TMEM lane quadrant this warp may read
+    int local = 0;
+    for (int w = blockIdx.x; w < n_work; w += gridDim.x, ++local) {
+      const int4 it = __ldg(work + w);
+      const int as = local & 1;
+      const uint32_t aphase = (local >> 1) & 1u;
+      if (!mbar_wait(tfull_bar(as), aphase, s_abort, status)) goto done;
+      tc_fence_after();
+      const int r = q * 32 + lane;
+      const bool row_ok = r < it.y;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + as * BN;
+      if (PHASE == 1) {
+        bf16* dst = out + (size_t)(it.x + r) * ld_out + it.w * 128;
+        const int n_left = n_out - it.w * 128;
+#pragma unroll 1
+        for (int c0 = 0; c0 < 128; c0 += 16) {
+          uint32_t g[16], u[16];
+          tmem_ld16(taddr + c0, g);
+          tmem_ld16(taddr + 128 + c0, u);
+          tmem_ld_wait();
+          uint4 o0, o1;
+          o0.x = pack_bf16(silu_mul(g[0], u[0]), silu_mul(g[1], u[1]));
+          o0.y = pack_bf16(silu_mul(g[2], u[2]), silu_mul(g[3], u[3]));
+          o0.z = pack_bf16(silu_mul(g[4], u[4]), silu_mul(g[5], u[5]));
+          o0.w = pack_bf16(silu_mul(g[6], u[6]), silu_mul(g[7], u[7]));
+          o1.x = pack_bf16(silu_mul(g[8], u[8]), silu_mul(g[9], u[9]));
+          o1.y = pack_bf16(silu_mul(g[10], u[10]), silu_mul(g[11], u[11]));
+          o1.z = pack_bf16(silu_mul(g[12], u[12]), silu_mul(g[13], u[13]));
+          o1.w = pack_bf16(silu_mul(g[14], u[14]), silu_mul(g[15], u[15]));
+          if (row_ok && c0 < n_left) *reinterpret_cast<uint4*>(dst + c0) = o0;
+          if (row_ok && c0 + 8 < n_left) *reinterpret_cast<uint4*>(dst + c0 + 8) = o1;
+        }
+      } else {
+        bf16* dst = out + (size_t)(it.x + r) * ld_out + it.w * BN;
+        const int n_left = n_out - it.w * BN;
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          uint32_t a[16], b[16];
+          tmem_ld16(taddr + c0, a);
+          tmem_ld16(taddr + c0 + 16, b);
+          tmem_ld_wait();
+          uint4 o[4];
+          o[0].x = pack_bf16(__uint_as_float(a[0]), __uint_as_float(a[1]));
+          o[0].y = pack_bf16(__uint_as_float(a[2]), __uint_as_float(a[3]));
+          o[0].z = pack_bf16(__uint_as_float(a[4]), __uint_as_float(a[5]));
+          o[0].w = pack_bf16(__uint_as_float(a[6]), __uint_as_float(a[7]));
+          o[1].x = pack_bf16(__uint_as_float(a[8]), __uint_as_float(a[9]));
+          o[1].y = pack_bf16(__uint_as_float(a[10]), __uint_as_float(a[11]));
+          o[1].z = pack_bf16(__uint_as_float(a[12]), __uint_as_float(a[13]));
+          o[1].w = pack_bf16(__uint_as_float(a[14]), __uint_as_float(a[15]));
+          o[2].x = pack_bf16(__uint_as_float(b[0]), __uint_as_float(b[1]));
+          o[2].y = pack_bf16(__uint_as_float(b[2]), __uint_as_float(b[3]));
+          o[2].z = pack_bf16(__uint_as_float(b[4]), __uint_as_float(b[5]));
+          o[2].w = pack_bf16(__uint_as_float(b[6]), __uint_as_float(b[7]));
+          o[3].x = pack_bf16(__uint_as_float(b[8]), __uint_as_float(b[9]));
+          o[3].y = pack_bf16(__uint_as_float(b[10]), __uint_as_float(b[11]));
+          o[3].z = pack_bf16(__uint_as_float(b[12]), __uint_as_float(b[13]));
+          o[3].w = pack_bf16(__uint_as_float(b[14]), __uint_as_float(b[15]));
+#pragma unroll
+          for (int v = 0; v < 4; ++v)
+            if (row_ok && c0 + 8 * v < n_left) *reinterpret_cast<uint4*>(dst + c0 + 8 * v) = o[v];
+        }
+      }
+      // all TMEM reads of this warp are complete (wait::ld above): hand the accumulator back
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(as));
+    }
+  }
+
+done:
+  if (*s_abort) {
+    // give copies and MMAs in flight time to land before shared memory and TMEM go away
+    for (int i = 0; i < 200; ++i) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---- tile list construction ------------------------------------------------------------------
+// plan: per group of the requested range, number of 128-row tiles; exclusive scan; totals.
+__global__ void __launch_bounds__(1024)
+plan_kernel(const int32_t* __restrict__ group_off, const int32_t* __restrict__ step_meta, int device, int nt1, int nt2,
+            int32_t* __restrict__ mtile_pref, int32_t* __restrict__ work_count) {
+  __shared__ int s_warp[32];
+  __shared__ int s_carry;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int G = step_meta[1];
+  const int g0 = device < 0 ? 0 : step_meta[3 + device];
+  const int g1 = device < 0 ? G : step_meta[3 + device + 1];
+  const int ng = g1 - g0;
+  if (tid == 0) s_carry = 0;
+  __syncthreads();
+  for (int b = 0; b < ng; b += 1024) {
+    int i = b + tid;
+    int v = 0;
+    if (i < ng) v = (group_off[g0 + i + 1] - group_off[g0 + i] + BM - 1) / BM;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int n = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += n;
+    }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      int wv = s_warp[lane], wi = wv;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        int n = __shfl_up_sync(0xffffffffu, wi, o);
+        if (lane >= o) wi += n;
+      }
+      s_warp[lane] = wi - wv;
+    }
+    __syncthreads();
+    int excl = s_carry + s_warp[warp] + incl - v;
+    if (i < ng) mtile_pref[i] = excl;
+    __syncthreads();
+    if (tid == 1023) s_carry = excl + v;
+    __syncthreads();
+  }
+  if (tid == 0) {
+    int mt = s_carry;
+    mtile_pref[ng] = mt;
+    work_count[0] = mt * nt1;
+    work_count[1] = mt * nt2;
+    work_count[2] = mt;
+    work_count[3] = g0;
+    work_count[4] = ng;
+  }
+}
+
+// fill: one thread per tile; tiles of a group are ordered n-tile major, m-tile minor.
+__global__ void __launch_bounds__(256)
+fill_kernel(const int32_t* __restrict__ group_off, const int32_t* __restrict__ group_w,
+            const int32_t* __restrict__ mtile_pref, const int32_t* __restrict__ work_count, int nt1, int nt2,
+            int max1, int max2, int4* __restrict__ work1, int4* __restrict__ work2) {
+  const int w1 = work_count[0], w2 = work_count[1], g0 = work_count[3], ng = work_count[4];
+  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < w1 + w2; idx += gridDim.x * blockDim.x) {
+    const bool first = idx < w1;
+    const int local = first ? idx : idx - w1;
+    const int nt = first ? nt1 : nt2;
+    const int mt_index = local / nt;  // position in units of "m-tiles x nt": find group by m-tile prefix
+    // largest gi with mtile_pref[gi] * nt <= local  <=>  mtile_pref[gi] <= local / nt
+    int lo = 0, hi = ng - 1;
+    while (lo < hi) {
+      int mid = (lo + hi + 1) >> 1;
+      if (mtile_pref[mid] <= mt_index) lo = mid; else hi = mid - 1;
+    }
+    // skip past empty groups that share the same prefix value: take the last group with that prefix
+    const int gi = lo;
+    const int mt_g = mtile_pref[gi + 1] - mtile_pref[gi];
+    const int rem = local - mtile_pref[gi] * nt;
+    const int n = rem / mt_g, m = rem % mt_g;
+    const int g = g0 + gi;
+    const int row0 = group_off[g] + m * BM;
+    int4 it;
+    it.x = row0;
+    it.y = min(BM, group_off[g + 1] - row0);
+    it.z = group_w[g];
+    it.w = n;
+    if (first) {
+      if (local < max1) work1[local] = it;
+    } else {
+      if (local < max2) work2[local] = it;
+    }
+  }
+}
+
+// ---- host side ---------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+// bf16 tensor [d2][d1][d0] (d0 innermost), box {b0, b1, 1}, 128-byte swizzle, zero fill out of bounds
+bool make_map(CUtensorMap* m, const void* ptr, uint64_t d0, uint64_t d1, uint64_t d2, uint32_t b0, uint32_t b1) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {d0, d1, d2};
+  cuuint64_t strides[2] = {d0 * 2, d0 * d1 * 2};
+  cuuint32_t box[3] = {b0, b1, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  int rank = d2 > 0 ? 3 : 2;
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+eb_status ebi_ffn_bind(eb_ctx* c) {
+  const eb_config& g = c->cfg;
+  const uint64_t nw = (uint64_t)g.L * (g.E + g.S);
+  if (!make_map(&c->tm_gate, c->w_gate, g.H, g.I, nw, BK, 128) ||
+      !make_map(&c->tm_up, c->w_up, g.H, g.I, nw, BK, 128) ||
+      !make_map(&c->tm_down, c->w_down, g.I, g.H, nw, BK, BN))
+    return ebi_fail(c, EB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the weights");
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e1 = cudaFuncSetAttribute(ffn_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    cudaError_t e2 = cudaFuncSetAttribute(ffn_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e1 != cudaSuccess || e2 != cudaSuccess) return ebi_check_cuda(c, e1 != cudaSuccess ? e1 : e2, "cudaFuncSetAttribute");
+    attr_set = true;
+  }
+  return EB_OK;
+}
+
+eb_status ebi_ffn_run(eb_ctx* c, cudaStream_t st, const void* xp, const int32_t* group_off, const int32_t* group_w,
+                      const int32_t* step_meta, void* yp, int32_t device) {
+  if (!xp || !group_off || !group_w || !step_meta || !yp) return ebi_fail(c, EB_ERR_INVALID_ARG, "null pointer");
+  if (!ebi_aligned16(xp) || !ebi_aligned16(yp)) return ebi_fail(c, EB_ERR_INVALID_ARG, "xp / yp must be 16-byte aligned");
+  if (!c->w_gate) return ebi_fail(c, EB_ERR_INVALID_ARG, "weights not bound");
+  if (!c->ws) return ebi_fail(c, EB_ERR_WORKSPACE, "no workspace set");
+  const eb_config& g = c->cfg;
+  const int rows = ebi_rows_cap(c);
+  CUtensorMap tm_x, tm_xs, tm_a, tm_as;
+  if (!make_map(&tm_x, xp, g.H, rows, 0, BK, BM) || !make_map(&tm_xs, xp, g.H, rows, 0, BK, kSmallRows) ||
+      !make_map(&tm_a, c->act, g.I, rows, 0, BK, BM) || !make_map(&tm_as, c->act, g.I, rows, 0, BK, kSmallRows))
+    return ebi_fail(c, EB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the activations");
+  const int nt1 = (g.I + 127) / 128, nt2 = (g.H + BN - 1) / BN;
+  {
+    KernelTimer timer(c, EBK_FFN_PLAN, st);
+    plan_kernel<<<1, 1024, 0, st>>>(group_off, step_meta, device, nt1, nt2, c->mtile_pref, c->work_count);
+  }
+  {
+    KernelTimer timer(c, EBK_FFN_FILL, st);
+    fill_kernel<<<c->num_sms, 256, 0, st>>>(group_off, group_w, c->mtile_pref, c->work_count, nt1, nt2, c->max_work1,
+                                            c->max_work2, c->work1, c->work2);
+  }
+  {
+    KernelTimer timer(c, EBK_FFN_GATEUP, st);
+    ffn_kernel<1><<<c->num_sms, kThreads, kSmemBytes, st>>>(tm_x, tm_xs, c->tm_gate, c->tm_up, c->work1, c->work_count,
+                                                            c->act, g.I, g.I, g.H, c->d_status);
+  }
+  {
+    KernelTimer timer(c, EBK_FFN_DOWN, st);
+    ffn_kernel<2><<<c->num_sms, kThreads, kSmemBytes, st>>>(tm_a, tm_as, c->tm_down, c->tm_down, c->work2, c->work_count,
+                                                            (bf16*)yp, g.H, g.H, g.I, c->d_status);
+  }
+  EB_LAUNCH_CHECK(c, "expert_ffn");
+  return EB_OK;
+}

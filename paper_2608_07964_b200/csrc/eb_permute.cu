@@ -1,0 +1,337 @@
+// eb_permute: dispatch on one GPU (Section 2.2) as a deterministic, stable counting sort of the
+// (token, expert) assignments of the chosen micro-batches by (virtual device, layer, expert),
+// followed by a 16-byte-vector gather of the token rows.
+//
+// Tokens are cut into chunks of <= 32 consecutive tokens of one micro-batch (one warp each).
+//   hist   : per chunk, assignments per expert                     -> chunk_hist[chunk][E]
+//   sizes  : per group, a warp scans the chunks of its layer in token order, leaving each
+//            chunk's first rank inside the group                   -> chunk_base, group_size
+//   scan   : exclusive prefix sum over groups                      -> group_off, group_w, step_meta
+//   rank   : per chunk, ranks by warp match (in assignment order)  -> pos, row_src
+//   gather : one warp per token reads the row once and writes it to its K + S rows.
+// No order-dependent atomics anywhere: rows inside a group are in (micro-batch, token) order.
+#include "eb_internal.cuh"
+
+namespace {
+
+constexpr int kWarps = 8;
+
+struct StepShape {
+  int nl;                       // active layers
+  int act_layer[EB_MAX_MB];     // ascending
+  int rank_of_mb[EB_MAX_MB];    // rank of the micro-batch's layer among active layers, -1 if not chosen
+};
+
+__device__ __forceinline__ StepShape step_shape(const BatchParams& bp, uint32_t run) {
+  StepShape s;
+  s.nl = 0;
+  // insertion of distinct layers in ascending order (n_mb <= 16)
+  for (int j = 0; j < bp.n_mb; ++j) {
+    if (!((run >> j) & 1u)) continue;
+    int l = bp.layer[j], p = 0;
+    bool dup = false;
+    for (int i = 0; i < s.nl; ++i) {
+      if (s.act_layer[i] == l) dup = true;
+      if (s.act_layer[i] < l) p = i + 1;
+    }
+    if (dup) continue;
+    for (int i = s.nl; i > p; --i) s.act_layer[i] = s.act_layer[i - 1];
+    s.act_layer[p] = l;
+    ++s.nl;
+  }
+  for (int j = 0; j < EB_MAX_MB; ++j) {
+    s.rank_of_mb[j] = -1;
+    if (j < bp.n_mb && ((run >> j) & 1u))
+      for (int i = 0; i < s.nl; ++i)
+        if (s.act_layer[i] == bp.layer[j]) s.rank_of_mb[j] = i;
+  }
+  return s;
+}
+
+// first token (local index) of micro-batch of T tokens whose home device is >= d
+__device__ __forceinline__ int home_start(int d, int T, int D) { return (int)(((long long)d * T + D - 1) / D); }
+
+// group id of (device d, active-layer rank lr, local slot) ; local slot < n_d + S
+__device__ __forceinline__ int group_id(const ModelParams& mp, int nl, int d, int lr, int local) {
+  int n_d = mp.dev_off[d + 1] - mp.dev_off[d];
+  return nl * (mp.dev_off[d] + d * mp.S) + lr * (n_d + mp.S) + local;
+}
+
+__device__ __forceinline__ int mb_of_chunk(const BatchParams& bp, int c) {
+  int j = 0;
+  while (j + 1 < bp.n_mb && c >= bp.chunk_off[j + 1]) ++j;
+  return j;
+}
+
+// ---- hist ----------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kWarps * 32)
+hist_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ res,
+            const int32_t* __restrict__ topk_idx, int32_t* __restrict__ chunk_hist) {
+  __shared__ int s_hist[kWarps][EB_MAX_E];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int c = blockIdx.x * kWarps + warp;
+  if (c >= bp.n_chunks) return;
+  const int E = mp.E, K = mp.K;
+  const int j = mb_of_chunk(bp, c);
+  const uint32_t run = res->run_mask;
+  int* h = s_hist[warp];
+  for (int e = lane; e < E; e += 32) h[e] = 0;
+  __syncwarp();
+  if ((run >> j) & 1u) {
+    int t0 = bp.tok_off[j] + (c - bp.chunk_off[j]) * 32;
+    int nt = min(32, bp.tok_off[j + 1] - t0);
+    for (int a = lane; a < nt * K; a += 32) atomicAdd(&h[topk_idx[(size_t)t0 * K + a]], 1);
+  }
+  __syncwarp();
+  for (int e = lane; e < E; e += 32) chunk_hist[(size_t)c * E + e] = h[e];
+}
+
+// ---- sizes ---------------------------------------------------------------------------------
+// One warp per group.  Routed group (d, lr, e): walks the chunks of the chosen micro-batches
+// sitting at that layer in token order; writes the running count before each chunk and the total.
+__global__ void __launch_bounds__(kWarps * 32)
+sizes_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ res,
+             const int32_t* __restrict__ chunk_hist, int32_t* __restrict__ chunk_base,
+             int32_t* __restrict__ group_size) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int g = blockIdx.x * kWarps + warp;
+  const uint32_t run = res->run_mask;
+  const StepShape ss = step_shape(bp, run);
+  const int G = ss.nl * (mp.E + mp.D * mp.S);
+  if (g >= G) return;
+  // decode g -> (d, lr, local)
+  int d = 0;
+  while (d + 1 < mp.D && g >= ss.nl * (mp.dev_off[d + 1] + (d + 1) * mp.S)) ++d;
+  const int n_d = mp.dev_off[d + 1] - mp.dev_off[d];
+  const int rel = g - ss.nl * (mp.dev_off[d] + d * mp.S);
+  const int lr = rel / (n_d + mp.S), local = rel % (n_d + mp.S);
+  if (local >= n_d) {
+    // shared expert: rows = chosen tokens at this layer whose home device is d (closed form)
+    if (lane == 0) {
+      int tot = 0;
+      for (int j = 0; j < bp.n_mb; ++j)
+        if (ss.rank_of_mb[j] == lr) {
+          int T = bp.tok_off[j + 1] - bp.tok_off[j];
+          tot += home_start(d + 1, T, mp.D) - home_start(d, T, mp.D);
+        }
+      group_size[g] = tot;
+    }
+    return;
+  }
+  const int e = mp.dev_list[mp.dev_off[d] + local];
+  int carry = 0;
+  for (int j = 0; j < bp.n_mb; ++j) {
+    if (ss.rank_of_mb[j] != lr) continue;
+    for (int c0 = bp.chunk_off[j]; c0 < bp.chunk_off[j + 1]; c0 += 32) {
+      int c = c0 + lane;
+      int v = c < bp.chunk_off[j + 1] ? chunk_hist[(size_t)c * mp.E + e] : 0;
+      int incl = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        int n = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += n;
+      }
+      if (c < bp.chunk_off[j + 1]) chunk_base[(size_t)c * mp.E + e] = carry + incl - v;
+      carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+  }
+  if (lane == 0) group_size[g] = carry;
+}
+
+// ---- scan ----------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024)
+scan_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ res,
+            const int32_t* __restrict__ group_size, int32_t* __restrict__ group_off,
+            int32_t* __restrict__ group_w, int32_t* __restrict__ step_meta) {
+  __shared__ int s_warp[32];
+  __shared__ int s_carry;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t run = res->run_mask;
+  const StepShape ss = step_shape(bp, run);
+  const int G = ss.nl * (mp.E + mp.D * mp.S);
+  if (tid == 0) s_carry = 0;
+  __syncthreads();
+  for (int base = 0; base < G; base += 1024) {
+    int g = base + tid;
+    int v = g < G ? group_size[g] : 0;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int n = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += n;
+    }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      int w = s_warp[lane], wi = w;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        int n = __shfl_up_sync(0xffffffffu, wi, o);
+        if (lane >= o) wi += n;
+      }
+      s_warp[lane] = wi - w;  // exclusive offset of each warp
+    }
+    __syncthreads();
+    int excl = s_carry + s_warp[warp] + incl - v;
+    if (g < G) {
+      group_off[g] = excl;
+      // weight matrix of the group
+      int d = 0;
+      while (d + 1 < mp.D && g >= ss.nl * (mp.dev_off[d + 1] + (d + 1) * mp.S)) ++d;
+      int n_d = mp.dev_off[d + 1] - mp.dev_off[d];
+      int rel = g - ss.nl * (mp.dev_off[d] + d * mp.S);
+      int lr = rel / (n_d + mp.S), local = rel % (n_d + mp.S);
+      int slot = local < n_d ? mp.dev_list[mp.dev_off[d] + local] : mp.E + (local - n_d);
+      group_w[g] = ss.act_layer[lr] * (mp.E + mp.S) + slot;
+    }
+    __syncthreads();
+    if (tid == 1023) s_carry = excl + v;
+    __syncthreads();
+  }
+  if (tid == 0) {
+    group_off[G] = s_carry;
+    step_meta[0] = s_carry;
+    step_meta[1] = G;
+    step_meta[2] = ss.nl;
+    for (int d = 0; d <= mp.D; ++d)
+      step_meta[3 + d] = d < mp.D ? ss.nl * (mp.dev_off[d] + d * mp.S) : G;
+    for (int i = 4 + mp.D; i < EB_META_LEN; ++i) step_meta[i] = 0;
+  }
+}
+
+// ---- rank ----------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kWarps * 32)
+rank_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ res,
+            const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ chunk_base,
+            const int32_t* __restrict__ group_off, int32_t* __restrict__ pos, int32_t* __restrict__ row_src) {
+  __shared__ int s_next[kWarps][EB_MAX_E];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int c = blockIdx.x * kWarps + warp;
+  if (c >= bp.n_chunks) return;
+  const int E = mp.E, K = mp.K, S = mp.S, KS = K + S;
+  const int j = mb_of_chunk(bp, c);
+  const uint32_t run = res->run_mask;
+  const int t0 = bp.tok_off[j] + (c - bp.chunk_off[j]) * 32;
+  const int nt = min(32, bp.tok_off[j + 1] - t0);
+  if (!((run >> j) & 1u)) {
+    for (int a = lane; a < nt * KS; a += 32) pos[(size_t)t0 * KS + a] = -1;
+    return;
+  }
+  const StepShape ss = step_shape(bp, run);
+  const int lr = ss.rank_of_mb[j];
+  int* next = s_next[warp];
+  for (int e = lane; e < E; e += 32) {
+    int d = mp.e2d[e];
+    next[e] = group_off[group_id(mp, ss.nl, d, lr, mp.e_local[e])] + chunk_base[(size_t)c * E + e];
+  }
+  __syncwarp();
+  // routed slots, in assignment order a = t_local * K + k
+  for (int a0 = 0; a0 < nt * K; a0 += 32) {
+    int a = a0 + lane;
+    bool valid = a < nt * K;
+    int e = valid ? topk_idx[(size_t)t0 * K + a] : -1 - lane;  // distinct dummies never match
+    unsigned peers = __match_any_sync(0xffffffffu, e);
+    int before = __popc(peers & ((1u << lane) - 1u));
+    int p = 0;
+    if (valid) {
+      p = next[e] + before;
+      int t = t0 + a / K, k = a % K;
+      pos[(size_t)t * KS + k] = p;
+      row_src[p] = t;
+    }
+    __syncwarp();
+    if (valid && before == 0) next[e] += __popc(peers);
+    __syncwarp();
+  }
+  // shared slots: closed-form rows
+  if (S > 0 && lane < nt) {
+    const int T = bp.tok_off[j + 1] - bp.tok_off[j];
+    const int tl = t0 + lane - bp.tok_off[j];
+    const int d = (int)(((long long)tl * mp.D) / T);
+    int before = 0;
+    for (int j2 = 0; j2 < j; ++j2)
+      if (ss.rank_of_mb[j2] == lr) {
+        int T2 = bp.tok_off[j2 + 1] - bp.tok_off[j2];
+        before += home_start(d + 1, T2, mp.D) - home_start(d, T2, mp.D);
+      }
+    const int n_d = mp.dev_off[d + 1] - mp.dev_off[d];
+    for (int s = 0; s < S; ++s) {
+      int p = group_off[group_id(mp, ss.nl, d, lr, n_d + s)] + before + (tl - home_start(d, T, mp.D));
+      pos[(size_t)(t0 + lane) * KS + K + s] = p;
+      row_src[p] = t0 + lane;
+    }
+  }
+}
+
+// ---- gather --------------------------------------------------------------------------------
+// One warp per token: the row is read once as 16-byte vectors and written to each of its rows.
+__global__ void __launch_bounds__(kWarps * 32)
+gather_kernel(int n_tok, int H, int KS, const uint4* __restrict__ x, const int32_t* __restrict__ pos,
+              uint4* __restrict__ xp) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int t = blockIdx.x * kWarps + warp;
+  if (t >= n_tok) return;
+  int my_pos = lane < KS ? pos[(size_t)t * KS + lane] : -1;
+  if (__shfl_sync(0xffffffffu, my_pos, 0) < 0) return;  // micro-batch does not run
+  const int vec = H / 8;                                // 16-byte vectors per row
+  const uint4* src = x + (size_t)t * vec;
+  for (int v0 = 0; v0 < vec; v0 += 32 * 4) {
+    uint4 r[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      int v = v0 + u * 32 + lane;
+      if (v < vec) r[u] = __ldg(src + v);
+    }
+    for (int s = 0; s < KS; ++s) {
+      int p = __shfl_sync(0xffffffffu, my_pos, s);
+      uint4* dst = xp + (size_t)p * vec;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        int v = v0 + u * 32 + lane;
+        if (v < vec) dst[v] = r[u];
+      }
+    }
+  }
+}
+
+}  // namespace
+
+extern "C" eb_status eb_permute(eb_ctx* c, void* stream, const eb_batch* batch, const eb_sched_result* d_res,
+                                const void* x, const int32_t* topk_idx, int32_t* group_off, int32_t* group_w,
+                                int32_t* row_src, int32_t* pos, void* xp, int32_t* step_meta) {
+  if (!c) return EB_ERR_INVALID_ARG;
+  BatchParams bp;
+  eb_status s = ebi_make_batch(c, batch, &bp);
+  if (s != EB_OK) return s;
+  if (!d_res || !x || !topk_idx || !group_off || !group_w || !row_src || !pos || !xp || !step_meta)
+    return ebi_fail(c, EB_ERR_INVALID_ARG, "null pointer");
+  if (!ebi_aligned16(x) || !ebi_aligned16(xp)) return ebi_fail(c, EB_ERR_INVALID_ARG, "x / xp must be 16-byte aligned");
+  if (!c->ws) return ebi_fail(c, EB_ERR_WORKSPACE, "no workspace set");
+  cudaStream_t st = (cudaStream_t)stream;
+  const int gcap = ebi_groups_cap(c);
+  const int chunk_blocks = (bp.n_chunks + kWarps - 1) / kWarps;
+  if (bp.n_chunks > 0) {
+    KernelTimer timer(c, EBK_PERMUTE_HIST, st);
+    hist_kernel<<<chunk_blocks, kWarps * 32, 0, st>>>(c->mp, bp, d_res, topk_idx, c->chunk_hist);
+  }
+  {
+    KernelTimer timer(c, EBK_PERMUTE_SIZES, st);
+    sizes_kernel<<<(gcap + kWarps - 1) / kWarps, kWarps * 32, 0, st>>>(c->mp, bp, d_res, c->chunk_hist, c->chunk_base,
+                                                                        c->group_size);
+  }
+  {
+    KernelTimer timer(c, EBK_PERMUTE_SCAN, st);
+    scan_kernel<<<1, 1024, 0, st>>>(c->mp, bp, d_res, c->group_size, group_off, group_w, step_meta);
+  }
+  if (bp.n_chunks > 0) {
+    KernelTimer timer(c, EBK_PERMUTE_RANK, st);
+    rank_kernel<<<chunk_blocks, kWarps * 32, 0, st>>>(c->mp, bp, d_res, topk_idx, c->chunk_base, group_off, pos, row_src);
+  }
+  if (bp.n_tok > 0) {
+    KernelTimer timer(c, EBK_PERMUTE_GATHER, st);
+    gather_kernel<<<(bp.n_tok + kWarps - 1) / kWarps, kWarps * 32, 0, st>>>(
+        bp.n_tok, c->cfg.H, c->cfg.K + c->cfg.S, (const uint4*)x, pos, (uint4*)xp);
+  }
+  EB_LAUNCH_CHECK(c, "permute");
+  return EB_OK;
+}

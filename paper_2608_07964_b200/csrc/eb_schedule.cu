@@ -1,0 +1,223 @@
+// eb_schedule: Schedule(S, m) of Algorithm 1 as one thread block.
+//
+// MaxUtil (Section 4.2) enumerates every subset of the pool with at least m members.  The pool
+// is split into a low and a high half; the summed load vector of each half-subset is tabulated
+// in shared memory (2 x 256 x D entries at most), so a subset costs D additions and a maximum.
+// Utilisation (Eq. 3 for one step) is sum(W) / (D * max(W)); D is common to all candidates, so
+// candidates are compared exactly by cross-multiplying sum and max in 64-bit integers.
+// Total order: higher utilisation, then more members, then the numerically smaller mask.
+// CumUtil / DiffPeak (Section 5.2) are sequential and run on one thread.
+#include "eb_internal.cuh"
+
+namespace {
+
+constexpr int kThreads = 1024;
+
+struct Cand {
+  long long num;   // sum_d W_d  (D if there is no work: U := 1)
+  long long peak;  // max_d W_d  (1 if there is no work)
+  int n;           // members
+  unsigned sub;    // subset in pool-relative bit positions (order preserving w.r.t. the real mask)
+};
+
+__device__ __forceinline__ bool better(const Cand& a, const Cand& b) {
+  if (b.n < 0) return a.n >= 0;
+  if (a.n < 0) return false;
+  long long l = a.num * b.peak, r = b.num * a.peak;
+  if (l != r) return l > r;
+  if (a.n != b.n) return a.n > b.n;
+  return a.sub < b.sub;
+}
+
+__device__ __forceinline__ Cand make_cand(const long long* w, int D, int n, unsigned sub) {
+  long long num = 0, peak = 0;
+  for (int d = 0; d < D; ++d) {
+    num += w[d];
+    peak = w[d] > peak ? w[d] : peak;
+  }
+  Cand c;
+  if (peak == 0) {
+    c.num = D;
+    c.peak = 1;
+  } else {
+    c.num = num;
+    c.peak = peak;
+  }
+  c.n = n;
+  c.sub = sub;
+  return c;
+}
+
+__global__ void __launch_bounds__(kThreads)
+schedule_kernel(int D, int n_mb, uint32_t pool_mask, int m, int policy, const int32_t* __restrict__ mb_load,
+                eb_sched_result* __restrict__ res) {
+  __shared__ int s_load[EB_MAX_MB][EB_MAX_D];
+  __shared__ int s_lo[256][EB_MAX_D];
+  __shared__ int s_hi[256][EB_MAX_D];
+  __shared__ int s_member[EB_MAX_MB];
+  __shared__ Cand s_best[kThreads / 32];
+  __shared__ uint32_t s_run;
+
+  const int tid = threadIdx.x;
+  for (int i = tid; i < EB_MAX_MB * EB_MAX_D; i += kThreads) {
+    int j = i / EB_MAX_D, d = i % EB_MAX_D;
+    s_load[j][d] = (j < n_mb && d < D) ? mb_load[j * D + d] : 0;
+  }
+  const int np = __popc(pool_mask);
+  if (tid == 0) {
+    int k = 0;
+    for (int j = 0; j < EB_MAX_MB; ++j)
+      if ((pool_mask >> j) & 1u) s_member[k++] = j;
+  }
+  __syncthreads();
+
+  if (np <= m || policy == EB_POLICY_ALL) {
+    if (tid == 0) s_run = pool_mask;
+  } else if (policy == EB_POLICY_MAXUTIL) {
+    const int nlo = np < 8 ? np : 8, nhi = np - nlo;
+    for (int i = tid; i < (1 << nlo) * EB_MAX_D; i += kThreads) {
+      int s = i / EB_MAX_D, d = i % EB_MAX_D, acc = 0;
+      for (int b = 0; b < nlo; ++b)
+        if ((s >> b) & 1) acc += s_load[s_member[b]][d];
+      s_lo[s][d] = acc;
+    }
+    for (int i = tid; i < (1 << nhi) * EB_MAX_D; i += kThreads) {
+      int s = i / EB_MAX_D, d = i % EB_MAX_D, acc = 0;
+      for (int b = 0; b < nhi; ++b)
+        if ((s >> b) & 1) acc += s_load[s_member[nlo + b]][d];
+      s_hi[s][d] = acc;
+    }
+    __syncthreads();
+    Cand best;
+    best.n = -1; best.num = 0; best.peak = 1; best.sub = 0;
+    const unsigned total = 1u << np, lomask = (1u << nlo) - 1u;
+    for (unsigned sub = tid + 1; sub < total; sub += kThreads) {
+      int n = __popc(sub);
+      if (n < m) continue;
+      long long w[EB_MAX_D];
+      const int* lo = s_lo[sub & lomask];
+      const int* hi = s_hi[sub >> nlo];
+#pragma unroll
+      for (int d = 0; d < EB_MAX_D; ++d) w[d] = (long long)lo[d] + hi[d];
+      Cand c = make_cand(w, D, n, sub);
+      if (better(c, best)) best = c;
+    }
+    // warp then block reduction under the total order
+    for (int o = 16; o > 0; o >>= 1) {
+      Cand oth;
+      oth.num = __shfl_xor_sync(0xffffffffu, best.num, o);
+      oth.peak = __shfl_xor_sync(0xffffffffu, best.peak, o);
+      oth.n = __shfl_xor_sync(0xffffffffu, best.n, o);
+      oth.sub = __shfl_xor_sync(0xffffffffu, best.sub, o);
+      if (better(oth, best)) best = oth;
+    }
+    if ((tid & 31) == 0) s_best[tid >> 5] = best;
+    __syncthreads();
+    if (tid == 0) {
+      Cand b = s_best[0];
+      for (int i = 1; i < kThreads / 32; ++i)
+        if (better(s_best[i], b)) b = s_best[i];
+      uint32_t mask = 0;
+      for (int k = 0; k < np; ++k)
+        if ((b.sub >> k) & 1u) mask |= 1u << s_member[k];
+      s_run = mask;
+    }
+  } else if (tid == 0) {
+    // CumUtil / DiffPeak: ascending pool members, the first always taken
+    long long w[EB_MAX_D];
+    for (int d = 0; d < EB_MAX_D; ++d) w[d] = s_load[s_member[0]][d];
+    uint32_t run = 1u << s_member[0];
+    int n = 1;
+    uint32_t peaks = 0;
+    auto peak_dev = [&](int j) {
+      int best = 0;
+      for (int d = 1; d < D; ++d)
+        if (s_load[j][d] > s_load[j][best]) best = d;
+      return best;
+    };
+    peaks |= 1u << peak_dev(s_member[0]);
+    for (int k = 1; k < np; ++k) {
+      int j = s_member[k];
+      bool take;
+      if (policy == EB_POLICY_CUMUTIL) {
+        long long w2[EB_MAX_D];
+        for (int d = 0; d < EB_MAX_D; ++d) w2[d] = w[d] + s_load[j][d];
+        Cand cur = make_cand(w, D, 0, 0), nxt = make_cand(w2, D, 0, 0);
+        take = nxt.num * cur.peak > cur.num * nxt.peak;
+      } else {
+        take = !((peaks >> peak_dev(j)) & 1u);
+      }
+      if (take) {
+        for (int d = 0; d < EB_MAX_D; ++d) w[d] += s_load[j][d];
+        run |= 1u << j;
+        peaks |= 1u << peak_dev(j);
+        ++n;
+      }
+    }
+    // top up to m members: repeatedly add the member whose inclusion gives the highest utilisation
+    while (n < m) {
+      int bj = -1;
+      Cand bu;
+      bu.n = -1; bu.num = 0; bu.peak = 1; bu.sub = 0;
+      for (int k = 0; k < np; ++k) {
+        int j = s_member[k];
+        if ((run >> j) & 1u) continue;
+        long long w2[EB_MAX_D];
+        for (int d = 0; d < EB_MAX_D; ++d) w2[d] = w[d] + s_load[j][d];
+        Cand cu = make_cand(w2, D, 0, 0);
+        if (bj < 0 || cu.num * bu.peak > bu.num * cu.peak) {
+          bj = j;
+          bu = cu;
+        }
+      }
+      if (bj < 0) break;
+      for (int d = 0; d < EB_MAX_D; ++d) w[d] += s_load[bj][d];
+      run |= 1u << bj;
+      ++n;
+    }
+    s_run = run;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    uint32_t run = s_run;
+    long long num = 0, peak = 0;
+    for (int d = 0; d < EB_MAX_D; ++d) {
+      long long v = 0;
+      for (int j = 0; j < EB_MAX_MB; ++j)
+        if ((run >> j) & 1u) v += s_load[j][d];
+      res->joint_load[d] = (int32_t)v;
+      num += v;
+      peak = v > peak ? v : peak;
+    }
+    res->run_mask = run;
+    res->defer_mask = pool_mask & ~run;
+    res->n_run = __popc(run);
+    res->status = EB_OK;
+    res->util_num = num;
+    res->util_den = (long long)D * peak;
+  }
+}
+
+}  // namespace
+
+extern "C" eb_status eb_schedule(eb_ctx* c, void* stream, const eb_batch* batch, int32_t m, eb_policy policy,
+                                 const int32_t* mb_load, eb_sched_result* d_res, eb_sched_result* h_res) {
+  if (!c) return EB_ERR_INVALID_ARG;
+  BatchParams bp;
+  eb_status s = ebi_make_batch(c, batch, &bp);
+  if (s != EB_OK) return s;
+  if (!mb_load || !d_res) return ebi_fail(c, EB_ERR_INVALID_ARG, "null pointer");
+  if (m < 1) return ebi_fail(c, EB_ERR_INVALID_ARG, "m must be at least 1");
+  if ((int)policy < 0 || (int)policy > EB_POLICY_ALL) return ebi_fail(c, EB_ERR_INVALID_ARG, "unknown policy");
+  cudaStream_t st = (cudaStream_t)stream;
+  {
+    KernelTimer timer(c, EBK_SCHEDULE, st);
+    schedule_kernel<<<1, kThreads, 0, st>>>(c->cfg.D, bp.n_mb, batch->pool_mask, m, (int)policy, mb_load, d_res);
+  }
+  EB_LAUNCH_CHECK(c, "schedule");
+  if (h_res) {
+    EB_CUDA(c, cudaMemcpyAsync(h_res, d_res, sizeof(eb_sched_result), cudaMemcpyDeviceToHost, st));
+    EB_CUDA(c, cudaStreamSynchronize(st));
+  }
+  return EB_OK;
+}

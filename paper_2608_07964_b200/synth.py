@@ -221,13 +221,15 @@ def zipf_bias(wl: Workload) -> np.ndarray:
     return tab.astype(np.float32)
 
 
-def logits_for(wl: Workload, mb: int, layer: int, device="cpu", bias: np.ndarray | None = None) -> torch.Tensor:
+def logits_for(wl: Workload, mb: int, layer: int, device="cpu", bias: np.ndarray | None = None,
+               T: int | None = None) -> torch.Tensor:
     """Router logits fp32 [T, E] of micro-batch `mb` when it sits at `layer`."""
     if bias is None:
         bias = zipf_bias(wl)
-    n = normal_f32(wl.seed, tensor_id(KIND_LOGIT, layer, mb), 0, wl.T * wl.E, 1.0, device)
+    T = wl.T if T is None else T
+    n = normal_f32(wl.seed, tensor_id(KIND_LOGIT, layer, mb), 0, T * wl.E, 1.0, device)
     b = torch.from_numpy(bias[layer]).to(device)
-    return n.view(wl.T, wl.E) + b
+    return n.view(T, wl.E) + b
 
 
 def packed_logits(wl: Workload, layers: Sequence[int] | None = None, device="cpu") -> torch.Tensor:
@@ -237,9 +239,10 @@ def packed_logits(wl: Workload, layers: Sequence[int] | None = None, device="cpu
     return torch.cat([logits_for(wl, j, layers[j], device, bias) for j in range(wl.N)], dim=0)
 
 
-def hidden_for(wl: Workload, mb: int, layer: int, device="cpu") -> torch.Tensor:
+def hidden_for(wl: Workload, mb: int, layer: int, device="cpu", T: int | None = None) -> torch.Tensor:
     """Hidden states bf16 [T, H] ~ N(0,1) of micro-batch `mb` entering `layer`."""
-    return normal_bf16(wl.seed, tensor_id(KIND_X, layer, mb), 0, wl.T * wl.H, 1.0, device).view(wl.T, wl.H)
+    T = wl.T if T is None else T
+    return normal_bf16(wl.seed, tensor_id(KIND_X, layer, mb), 0, T * wl.H, 1.0, device).view(T, wl.H)
 
 
 def packed_hidden(wl: Workload, layers: Sequence[int] | None = None, device="cpu") -> torch.Tensor:

@@ -1,0 +1,304 @@
+"""GPU parity: every stage of the cross-layer MoE step, called through the C ABI, against the CPU
+oracle on the same seeded inputs.  Integers (routing, schedule, loads, permutation) bit-exact;
+expert outputs within |gpu - ref| <= 2e-2 * max|ref| + 1e-3 elementwise (oracle in fp32 from the
+same bf16 weights)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import eb_oracle as O
+from paper_2608_07964_b200 import synth
+from tests import harness as Hn
+
+pytestmark = pytest.mark.gpu
+
+
+def _binding():
+    from paper_2608_07964_b200 import binding
+    return binding
+
+
+def _full_step(case, store, m, policy=O.POLICY_MAXUTIL, pool_mask=None, check_ffn=True, groups_to_check=None,
+               rows_per_group=None):
+    B = _binding()
+    wl = case.wl
+    n_mb = len(case.layers)
+    pool = ((1 << n_mb) - 1) if pool_mask is None else pool_mask
+    step = B.from_workload(wl, max_tokens=max(case.T_tot, 1))
+    step.bind_weights(store.gate, store.up, store.down)
+    T = case.T_tot
+    step.logits[:T].copy_(case.logits)
+    step.x[:T].copy_(case.x)
+    step.out.fill_(-7.0)
+    batch = B.Batch(case.tok_off, case.layers, pool)
+    step.eb_route(batch)
+    step.eb_schedule(batch, m, policy)
+    step.eb_permute(batch)
+    step.eb_expert_ffn_grouped()
+    step.eb_combine(batch)
+    torch.cuda.synchronize()
+    assert step.device_status() == 0
+
+    ref = Hn.oracle_front(case, pool, m, policy)
+    Hn.check_front(step, case, ref, n_mb)
+    if not check_ffn:
+        return step, ref
+    R = int(ref["group_off"][-1])
+    xp = step.xp[:R].float().cpu().numpy()
+    yp_gpu = step.yp[:R].float().cpu().numpy()
+    G = len(ref["group_w"])
+    if groups_to_check is None:
+        y_ref = O.expert_ffn(xp, ref["group_off"], ref["group_w"], store.get)
+        assert Hn.within_bar(yp_gpu, y_ref), f"expert outputs off by {Hn.worst(yp_gpu, y_ref):.2f} x bar"
+        out_ref, done = O.combine(y_ref, ref["pos"], ref["w"], wl.K, wl.S)
+        out_gpu = step.out[:T].float().cpu().numpy()
+        assert Hn.within_bar(out_gpu[done], out_ref[done]), f"aggregated output off by {Hn.worst(out_gpu[done], out_ref[done]):.2f} x bar"
+        assert (out_gpu[~done] == -7.0).all(), "rows of micro-batches that did not run must stay untouched"
+    else:
+        # sampled groups: the oracle computes whole groups (or their first rows) one by one
+        scale = 0.0
+        checked = []
+        for g in groups_to_check:
+            r0, r1 = int(ref["group_off"][g]), int(ref["group_off"][g + 1])
+            if rows_per_group:
+                r1 = min(r1, r0 + rows_per_group)
+            if r1 == r0:
+                continue
+            wg, wu, wd = store.get(int(ref["group_w"][g]))
+            y = O.swiglu_mlp(xp[r0:r1], wg, wu, wd)
+            checked.append((r0, r1, y))
+            scale = max(scale, float(np.abs(y).max()))
+        assert checked
+        for r0, r1, y in checked:
+            err = np.abs(yp_gpu[r0:r1].astype(np.float64) - y)
+            assert (err <= Hn.REL * scale + Hn.ABS).all(), f"group rows {r0}:{r1} off by {err.max() / (Hn.REL * scale + Hn.ABS):.2f} x bar"
+        # aggregation on sampled tokens from the library's own expert outputs (bf16), tight tolerance
+        rng = np.random.default_rng(0)
+        toks = [t for t in rng.choice(T, size=min(T, 64), replace=False) if ref["pos"][t, 0] >= 0]
+        yp32 = step.yp[:R].float().cpu().numpy()
+        out_ref, _ = O.combine(yp32, ref["pos"][toks], ref["w"][toks], wl.K, wl.S)
+        out_gpu = step.out[:T].float().cpu().numpy()[toks]
+        assert np.allclose(out_gpu, out_ref, rtol=1e-2, atol=1e-3 * max(1.0, np.abs(out_ref).max()))
+    return step, ref
+
+
+# ----------------------------------------------------------------------------------- full configs
+def test_c1_full_step_all_policies():
+    wl = synth.workload("c1")
+    store = Hn.WeightStore(wl)
+    case = Hn.make_case(wl)
+    for pol in (O.POLICY_MAXUTIL, O.POLICY_CUMUTIL, O.POLICY_DIFFPEAK, O.POLICY_ALL):
+        _full_step(case, store, wl.m, pol)
+
+
+def test_c1_not_renormalised_weights():
+    wl = synth.workload("c1", renorm_topk=0)
+    _full_step(Hn.make_case(wl), Hn.WeightStore(wl), wl.m)
+
+
+def test_c2_decode_shape_full_step():
+    wl = synth.workload("c2")
+    store = Hn.WeightStore(wl)
+    _full_step(Hn.make_case(wl), store, wl.m)
+
+
+def test_c3_fine_grained_sampled():
+    wl = synth.workload("c3")
+    store = Hn.WeightStore(wl)
+    case = Hn.make_case(wl)
+    ref = Hn.oracle_front(case, (1 << wl.N) - 1, wl.m, O.POLICY_MAXUTIL)
+    sizes = np.diff(ref["group_off"])
+    G = len(sizes)
+    order = np.argsort(sizes)
+    pick = sorted({0, G - 1, int(order[-1]), int(order[-2]), int(order[len(order) // 2]),
+                   *[int(g) for g in np.random.default_rng(1).choice(G, 12, replace=False)],
+                   *[g for g, (_, _, e) in enumerate(ref["groups"]) if e >= wl.E][:3]})
+    _full_step(case, store, wl.m, groups_to_check=pick)
+
+
+def test_c3_initial_state_sampled():
+    # Algorithm 1's first step: every micro-batch at layer 0 (large groups, many row tiles per group)
+    wl = synth.workload("c3", layers_override=tuple([0] * 16))
+    store = Hn.WeightStore(wl)
+    case = Hn.make_case(wl)
+    _full_step(case, store, wl.m, groups_to_check=[0, 7, 33, 65, 79], rows_per_group=300)
+
+
+def test_c4_large_experts_sampled():
+    wl = synth.workload("c4")
+    store = Hn.WeightStore(wl)
+    case = Hn.make_case(wl)
+    ref = Hn.oracle_front(case, (1 << wl.N) - 1, wl.m, O.POLICY_MAXUTIL)
+    sizes = np.diff(ref["group_off"])
+    nz = [int(g) for g in np.nonzero(sizes)[0]]
+    pick = sorted({nz[0], nz[-1], nz[len(nz) // 2], int(np.argmax(sizes))})
+    # rows from the start of each sampled group and, through rows_per_group, across a tile boundary
+    _full_step(case, store, wl.m, groups_to_check=pick, rows_per_group=160)
+
+
+# ----------------------------------------------------------------------------------- edge cases
+def _small(**kw):
+    base = dict(L=3, E=6, K=2, S=1, H=72, I=200, D=3, mapping="mod", N=4, T=8, zipf_s=1.0)
+    base.update(kw)
+    return synth.Workload(name="edge", **base)
+
+
+@pytest.mark.parametrize("tokens,layers,pool,m", [
+    ([5, 33, 0, 64], [0, 2, 1, 2], 0b1111, 3),       # ragged, an empty micro-batch, two sharing a layer
+    ([1, 2, 3, 4], [1, 1, 1, 1], 0b1111, 2),         # fewer tokens than devices, one layer only
+    ([40, 40, 40, 40], [0, 1, 2, 0], 0b0110, 1),     # pool is a strict subset
+    ([130, 7, 129, 31], [2, 2, 0, 1], 0b1011, 4),    # pool smaller than m: everything in the pool runs
+    ([16, 16, 16, 16], [0, 0, 0, 0], 0b0000, 2),     # empty pool: nothing runs
+])
+def test_edge_shapes(tokens, layers, pool, m):
+    wl = _small()
+    store = Hn.WeightStore(wl)
+    case = Hn.make_case(wl, tokens, layers)
+    _full_step(case, store, m, pool_mask=pool)
+
+
+def test_edge_k_equals_e_single_device_no_shared():
+    wl = _small(E=4, K=4, S=0, D=1, H=64, I=64)
+    _full_step(Hn.make_case(wl, [9, 70, 3, 20], [0, 1, 2, 1]), Hn.WeightStore(wl), 3)
+
+
+def test_edge_max_micro_batches_and_wide_router():
+    wl = _small(L=5, E=200, K=8, S=2, D=16, N=16, T=12, H=128, I=136, mapping="mod")
+    case = Hn.make_case(wl, [12 + (j % 5) for j in range(16)], [(j * 5) // 16 for j in range(16)])
+    _full_step(case, Hn.WeightStore(wl), 12)
+
+
+def test_multi_tile_groups_and_tails():
+    # groups of several hundred rows: more than one 128-row tile per group, ragged last tiles,
+    # output widths that are not multiples of the tile widths
+    wl = _small(L=2, E=4, K=2, S=1, D=2, N=2, T=700, H=264, I=328, mapping="contiguous", zipf_s=0.5)
+    _full_step(Hn.make_case(wl, [700, 519], [0, 0]), Hn.WeightStore(wl), 2)
+
+
+# ----------------------------------------------------------------------------------- schedule alone
+def test_schedule_random_load_matrices_bit_exact():
+    B = _binding()
+    rng = np.random.default_rng(12345)
+    wl = _small(D=5)
+    step = B.from_workload(wl, max_tokens=64)
+    n_checked = 0
+    for trial in range(2500):
+        n_mb = int(rng.integers(1, 9)) if trial % 50 else 16
+        D = 5
+        hi = [3, 30, 5000][trial % 3]
+        loads = rng.integers(0, hi, size=(n_mb, D)).astype(np.int32)
+        if trial % 7 == 0:
+            loads[rng.integers(0, n_mb)] = 0
+        pool = int(rng.integers(0, 1 << n_mb))
+        m = int(rng.integers(1, n_mb + 1))
+        dev_loads = torch.zeros((16, D), dtype=torch.int32, device="cuda")
+        dev_loads[:n_mb] = torch.from_numpy(loads).cuda()
+        batch = B.Batch([0] * (n_mb + 1), [0] * n_mb, pool)
+        for pol in (O.POLICY_MAXUTIL, O.POLICY_CUMUTIL, O.POLICY_DIFFPEAK, O.POLICY_ALL):
+            if n_mb == 16 and pol == O.POLICY_MAXUTIL and trial % 200:
+                continue
+            got = step.eb_schedule(batch, m, pol, to_host=True, mb_load=dev_loads)
+            ref = O.schedule(loads, pool, m, pol)
+            for k in ("run_mask", "defer_mask", "n_run", "joint_load", "util_num", "util_den"):
+                assert got[k] == ref[k], (trial, pol, k, got[k], ref[k], loads.tolist(), pool, m)
+            n_checked += 1
+    assert n_checked > 9000
+
+
+# ----------------------------------------------------------------------------------- combine alone
+def test_combine_alone_with_oracle_expert_outputs():
+    B = _binding()
+    wl = synth.workload("c1")
+    case = Hn.make_case(wl)
+    store = Hn.WeightStore(wl)
+    step, ref = _full_step(case, store, wl.m, check_ffn=False)
+    R = int(ref["group_off"][-1])
+    xp = step.xp[:R].float().cpu().numpy()
+    y = O.expert_ffn(xp, ref["group_off"], ref["group_w"], store.get)
+    y_bf = torch.from_numpy(y).to(torch.bfloat16)
+    step.yp[:R].copy_(y_bf)
+    batch = B.Batch(case.tok_off, case.layers)
+    step.eb_combine(batch)
+    out_ref, done = O.combine(y_bf.float().numpy(), ref["pos"], ref["w"], wl.K, wl.S)
+    out = step.out[:case.T_tot].float().cpu().numpy()
+    # only the final bf16 rounding and fp32 summation order separate the two
+    assert np.allclose(out[done], out_ref[done], rtol=2 ** -7, atol=1e-6)
+
+
+# ----------------------------------------------------------------------------------- per-device pass
+def test_per_device_pass_covers_exactly_its_rows():
+    B = _binding()
+    wl = synth.workload("c1")
+    case = Hn.make_case(wl)
+    store = Hn.WeightStore(wl)
+    step, ref = _full_step(case, store, wl.m)
+    R = int(ref["group_off"][-1])
+    full = step.yp[:R].clone()
+    firsts = step.meta()["dev_group_off"]
+    for d in range(wl.D):
+        step.yp.fill_(3.0)
+        step.eb_expert_ffn_grouped(device=d)
+        torch.cuda.synchronize()
+        r0, r1 = int(ref["group_off"][firsts[d]]), int(ref["group_off"][firsts[d + 1]])
+        assert torch.equal(step.yp[r0:r1], full[r0:r1])
+        assert (step.yp[:r0] == 3.0).all() and (step.yp[r1:R] == 3.0).all()
+    assert step.device_status() == 0
+
+
+# ----------------------------------------------------------------------------------- whole-step entry points
+def test_step_and_step_host_match_the_five_calls():
+    B = _binding()
+    wl = synth.workload("c1")
+    case = Hn.make_case(wl)
+    store = Hn.WeightStore(wl)
+    step, ref = _full_step(case, store, wl.m)
+    T = case.T_tot
+    want = step.out[:T].clone()
+    batch = B.Batch(case.tok_off, case.layers)
+    step.out.fill_(-7.0)      # rows of deferred micro-batches keep whatever the buffer held
+    step.eb_step(batch, wl.m)
+    torch.cuda.synchronize()
+    assert torch.equal(step.out[:T], want)
+    h_logits = case.logits.clone().pin_memory()
+    h_x = case.x.clone().pin_memory()
+    h_out = torch.full((T, wl.H), -7.0, dtype=torch.bfloat16).pin_memory()
+    res = step.eb_step_host(batch, wl.m, h_logits, h_x, h_out)
+    assert res["run_mask"] == ref["sched"]["run_mask"]
+    assert torch.equal(h_out, want.cpu())
+
+
+def test_deferred_micro_batch_keeps_its_routing():
+    B = _binding()
+    wl = synth.workload("c1")
+    case = Hn.make_case(wl)
+    step = B.from_workload(wl)
+    T = case.T_tot
+    step.logits[:T].copy_(case.logits)
+    batch = B.Batch(case.tok_off, case.layers)
+    step.eb_route(batch)
+    idx0, load0 = step.topk_idx.clone(), step.mb_load.clone()
+    step.logits[:T].copy_(torch.flip(case.logits, dims=[1]))       # new logits, but only micro-batch 1 is re-routed
+    step.eb_route(batch, route_mask=0b0010)
+    a, b = case.tok_off[1], case.tok_off[2]
+    assert torch.equal(step.topk_idx[:a], idx0[:a]) and torch.equal(step.topk_idx[b:T], idx0[b:T])
+    assert not torch.equal(step.topk_idx[a:b], idx0[a:b])
+    assert torch.equal(step.mb_load[[0, 2, 3]], load0[[0, 2, 3]])
+    assert int(step.mb_load[1].sum()) == (b - a) * wl.K
+
+
+def test_argument_errors_return_codes():
+    B = _binding()
+    wl = synth.workload("c1")
+    step = B.from_workload(wl)
+    batch = B.Batch([0, 10, 20], [0, 9])             # layer out of range
+    with pytest.raises(B.EbError) as e:
+        step.eb_route(batch)
+    assert e.value.code == 1
+    with pytest.raises(B.EbError):
+        step.eb_schedule(B.Batch([0, 10], [0]), 0)   # m < 1
+    with pytest.raises(B.EbError):
+        step.eb_route(B.Batch([0, 10000], [0]))      # more tokens than the context was sized for
+    with pytest.raises(B.EbError) as e:
+        step.eb_expert_ffn_grouped()                 # weights not bound
+    assert e.value.code == 1
+    assert step.device_status() == 0
