@@ -202,6 +202,37 @@ eb_status eb_step_host(eb_ctx* ctx, void* stream, const eb_batch* batch, uint32_
                        eb_policy policy, const eb_step_buffers* buf,
                        const float* h_logits, const void* h_x, void* h_out, eb_sched_result* h_res);
 
+/* ---- allocation-free variant --------------------------------------------------------------- */
+
+/* Largest packed token count eb_permute_noalloc accepts (its scratch is a fixed array). */
+enum { EB_NOALLOC_MAX_TOKENS = 4096 };
+
+/* The paper has no counterpart to this call; it exists for callers that are not allowed to
+ * create device allocations where they invoke the library: a serving process that has handed all
+ * free HBM to its cache and must not grow, a plug-in running inside a host framework's callback
+ * while that framework owns the allocator, a latency-critical loop that cannot take cudaMalloc's
+ * implicit synchronisation.  Such callers cannot use eb_create / eb_set_workspace.
+ *
+ * Computes exactly what eb_permute computes (same outputs, same layouts, same capacities of the
+ * output buffers: group_off [EB_MAX_MB*(E+D*S)+1], group_w [EB_MAX_MB*(E+D*S)],
+ * row_src [T_tot*(K+S)], pos [T_tot, K+S], xp [T_tot*(K+S), H], step_meta [EB_META_LEN]), but
+ * needs no context and no workspace.  The model shape comes in `cfg` (host; max_tokens and I are
+ * ignored) and the scratch (expert tables, per-chunk histograms, group sizes; about 316 KB) is a
+ * static device array inside the library, resident on every GPU that loads the library until
+ * the process exits.  It calls no cudaMalloc, cudaFree or other allocating routine.
+ *
+ * - At most EB_NOALLOC_MAX_TOKENS packed tokens; more returns EB_ERR_UNSUPPORTED and launches nothing.
+ * - The first call on each device resolves the array's device address (cudaGetSymbolAddress, with
+ *   that device current); make that first call outside any stream capture.
+ * - All calls on a device share the one array, which keeps the previous call's contents; the call
+ *   re-initialises what it reads (tables copied, counters cleared) on `stream`.  Two calls whose
+ *   work overlaps on the GPU (different streams, or different threads) race on it: serialise them.
+ * - `err` (host, may be NULL) receives a description of a failure, truncated to err_cap bytes. */
+eb_status eb_permute_noalloc(const eb_config* cfg, void* stream, const eb_batch* batch,
+                             const eb_sched_result* d_res, const void* x, const int32_t* topk_idx,
+                             int32_t* group_off, int32_t* group_w, int32_t* row_src, int32_t* pos,
+                             void* xp, int32_t* step_meta, char* err, size_t err_cap);
+
 /* ---- status and timing -------------------------------------------------------------------- */
 
 /* Reads (and clears) the context's device status word; synchronises the device. */

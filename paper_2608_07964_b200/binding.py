@@ -45,6 +45,7 @@ class EbStepBuffers(C.Structure):
 SYMBOLS = ["eb_create", "eb_destroy", "eb_bind_weights", "eb_workspace_bytes", "eb_set_workspace",
            "eb_rows_capacity", "eb_groups_capacity", "eb_route", "eb_schedule", "eb_permute",
            "eb_expert_ffn_grouped", "eb_expert_ffn_device", "eb_combine", "eb_step", "eb_step_host",
+           "eb_permute_noalloc",
            "eb_device_status", "eb_num_kernels", "eb_kernel_name", "eb_set_timing", "eb_kernel_ms",
            "eb_status_string", "eb_last_error"]
 
@@ -81,6 +82,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.eb_combine.argtypes = [vp, vp, C.POINTER(EbBatch), vp, vp, vp, vp, vp]
     lib.eb_step.argtypes = [vp, vp, C.POINTER(EbBatch), u32, i32, i32, C.POINTER(EbStepBuffers)]
     lib.eb_step_host.argtypes = [vp, vp, C.POINTER(EbBatch), u32, i32, i32, C.POINTER(EbStepBuffers), vp, vp, vp, vp]
+    lib.eb_permute_noalloc.argtypes = [C.POINTER(EbConfig), vp, C.POINTER(EbBatch), vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                       C.c_char_p, C.c_size_t]
     lib.eb_device_status.argtypes = [vp, C.POINTER(i32)]
     lib.eb_num_kernels.argtypes = []
     lib.eb_kernel_name.argtypes = [i32]
@@ -274,6 +277,24 @@ class MoEStep:
         arr = (C.c_float * n)()
         self._check(self.lib.eb_kernel_ms(self.ctx, arr))
         return {self.lib.eb_kernel_name(i).decode(): arr[i] for i in range(n) if arr[i] >= 0}
+
+
+def permute_noalloc(L, E, K, S, H, D, expert_to_device: Sequence[int], batch: Batch, sched: torch.Tensor,
+                    x: torch.Tensor, topk_idx: torch.Tensor, group_off: torch.Tensor, group_w: torch.Tensor,
+                    row_src: torch.Tensor, pos: torch.Tensor, xp: torch.Tensor, step_meta: torch.Tensor) -> None:
+    """eb_permute_noalloc: the dispatch step for callers that may not allocate device memory.
+
+    No context and no workspace: the library's built-in static scratch is used, which limits the
+    call to 4096 packed tokens.  All tensors are caller-owned device buffers."""
+    lib = load_library()
+    e2d = (C.c_int32 * E)(*expert_to_device)
+    cfg = EbConfig(L, E, K, S, H, 8, D, 1, batch.n_tok, e2d)
+    err = C.create_string_buffer(256)
+    code = lib.eb_permute_noalloc(C.byref(cfg), _stream(), C.byref(batch.c), sched.data_ptr(), x.data_ptr(),
+                                  topk_idx.data_ptr(), group_off.data_ptr(), group_w.data_ptr(), row_src.data_ptr(),
+                                  pos.data_ptr(), xp.data_ptr(), step_meta.data_ptr(), err, 256)
+    if code != 0:
+        raise EbError(code, lib.eb_status_string(code).decode() + ": " + err.value.decode())
 
 
 def _sched_dict(h: EbSchedResult, D: int) -> Dict:

@@ -10,6 +10,8 @@
 //   rank   : per chunk, ranks by warp match (in assignment order)  -> pos, row_src
 //   gather : one warp per token reads the row once and writes it to its K + S rows.
 // No order-dependent atomics anywhere: rows inside a group are in (micro-batch, token) order.
+#include <cstring>
+
 #include "eb_internal.cuh"
 
 namespace {
@@ -333,5 +335,127 @@ extern "C" eb_status eb_permute(eb_ctx* c, void* stream, const eb_batch* batch, 
         bp.n_tok, c->cfg.H, c->cfg.K + c->cfg.S, (const uint4*)x, pos, (uint4*)xp);
   }
   EB_LAUNCH_CHECK(c, "permute");
+  return EB_OK;
+}
+
+// ---- eb_permute_noalloc ------------------------------------------------------------------------
+// Same dispatch as eb_permute for callers that must not create device allocations: no context, no
+// workspace.  The expert tables and the permutation scratch live in one file-scope device array
+// that every GPU loading the library holds until the process exits.
+namespace {
+
+constexpr int kNaMaxTokens = EB_NOALLOC_MAX_TOKENS;
+constexpr int kNaMaxChunks = kNaMaxTokens / 32 + EB_MAX_MB;
+constexpr int kNaTableWords = 1024;                                   // e2d | dev_off | dev_list | e_local
+constexpr int kNaHistWords = kNaMaxChunks * EB_MAX_E;
+constexpr int kNaGroupWords = EB_MAX_MB * (EB_MAX_E + EB_MAX_D * EB_MAX_S);
+constexpr int kNaWords = kNaTableWords + 2 * kNaHistWords + kNaGroupWords;
+static_assert(3 * EB_MAX_E + EB_MAX_D + 1 <= kNaTableWords, "expert tables do not fit");
+
+// About 316 KB.  In host code this name is only a handle for cudaGetSymbolAddress, never a pointer.
+static __device__ __align__(256) int32_t g_noalloc_scratch[kNaWords];
+
+constexpr int kNaMaxDevices = 64;
+int32_t* g_noalloc_ptr[kNaMaxDevices] = {};
+
+eb_status noalloc_fail(char* err, size_t cap, eb_status s, const char* msg) {
+  if (err && cap) {
+    size_t n = strlen(msg) < cap - 1 ? strlen(msg) : cap - 1;
+    memcpy(err, msg, n);
+    err[n] = 0;
+  }
+  return s;
+}
+
+}  // namespace
+
+extern "C" eb_status eb_permute_noalloc(const eb_config* cfg, void* stream, const eb_batch* batch,
+                                        const eb_sched_result* d_res, const void* x, const int32_t* topk_idx,
+                                        int32_t* group_off, int32_t* group_w, int32_t* row_src, int32_t* pos,
+                                        void* xp, int32_t* step_meta, char* err, size_t err_cap) {
+  if (err && err_cap) err[0] = 0;
+  if (!cfg || !cfg->expert_to_device) return noalloc_fail(err, err_cap, EB_ERR_INVALID_ARG, "null config");
+  const eb_config& g = *cfg;
+  if (g.L < 1 || g.E < 1 || g.E > EB_MAX_E || g.K < 1 || g.K > EB_MAX_K || g.K > g.E || g.S < 0 || g.S > EB_MAX_S ||
+      g.D < 1 || g.D > EB_MAX_D || g.H < 8 || (g.H % 8))
+    return noalloc_fail(err, err_cap, EB_ERR_UNSUPPORTED, "shape outside the library limits");
+  for (int e = 0; e < g.E; ++e)
+    if (g.expert_to_device[e] < 0 || g.expert_to_device[e] >= g.D)
+      return noalloc_fail(err, err_cap, EB_ERR_INVALID_ARG, "expert_to_device entry out of range");
+  if (!batch || !batch->tok_off || !batch->layer) return noalloc_fail(err, err_cap, EB_ERR_INVALID_ARG, "null batch");
+  if (batch->n_mb >= 0 && batch->n_mb <= EB_MAX_MB && batch->tok_off[batch->n_mb] > kNaMaxTokens)
+    return noalloc_fail(err, err_cap, EB_ERR_UNSUPPORTED,
+                        "eb_permute_noalloc handles at most EB_NOALLOC_MAX_TOKENS (4096) packed tokens: "
+                        "its scratch is a fixed device array; use eb_permute with a workspace for more");
+  eb_ctx tmp;  // host-only helper for the shared argument checks; owns no device memory
+  tmp.cfg = g;
+  tmp.cfg.max_tokens = kNaMaxTokens;
+  BatchParams bp;
+  eb_status s = ebi_make_batch(&tmp, batch, &bp);
+  if (s != EB_OK) return noalloc_fail(err, err_cap, s, tmp.err.c_str());
+  if (!d_res || !x || !topk_idx || !group_off || !group_w || !row_src || !pos || !xp || !step_meta)
+    return noalloc_fail(err, err_cap, EB_ERR_INVALID_ARG, "null pointer");
+  if (!ebi_aligned16(x) || !ebi_aligned16(xp))
+    return noalloc_fail(err, err_cap, EB_ERR_INVALID_ARG, "x / xp must be 16-byte aligned");
+
+  // one-time set-up per device: resolve the device address of the scratch array
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNaMaxDevices)
+    return noalloc_fail(err, err_cap, EB_ERR_CUDA, "cudaGetDevice failed or device index too large");
+  if (!g_noalloc_ptr[dev]) {
+    int32_t* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress((void**)&p, g_noalloc_scratch);
+    if (e != cudaSuccess || !p) return noalloc_fail(err, err_cap, EB_ERR_CUDA, cudaGetErrorString(e));
+    g_noalloc_ptr[dev] = p;
+  }
+  int32_t* base = g_noalloc_ptr[dev];
+  int32_t* d_tab = base;
+  int32_t* d_hist = base + kNaTableWords;
+  int32_t* d_cbase = d_hist + kNaHistWords;
+  int32_t* d_gsize = d_cbase + kNaHistWords;
+
+  // expert tables, same layout as a context's: e2d | dev_off | dev_list | e_local
+  int32_t tab[kNaTableWords];
+  int32_t* h_off = tab + g.E;
+  int32_t* h_list = h_off + g.D + 1;
+  int32_t* h_local = h_list + g.E;
+  int n = 0;
+  for (int d = 0; d < g.D; ++d) {
+    h_off[d] = n;
+    for (int e = 0; e < g.E; ++e)
+      if (g.expert_to_device[e] == d) {
+        h_local[e] = n - h_off[d];
+        h_list[n++] = e;
+      }
+  }
+  h_off[g.D] = n;
+  for (int e = 0; e < g.E; ++e) tab[e] = g.expert_to_device[e];
+  ModelParams mp;
+  mp.L = g.L; mp.E = g.E; mp.K = g.K; mp.S = g.S; mp.H = g.H; mp.I = g.I; mp.D = g.D;
+  mp.renorm = g.renorm_topk ? 1 : 0;
+  mp.e2d = d_tab;
+  mp.dev_off = d_tab + g.E;
+  mp.dev_list = mp.dev_off + g.D + 1;
+  mp.e_local = mp.dev_list + g.E;
+
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t ce = cudaMemcpyAsync(d_tab, tab, sizeof(int32_t) * (3 * g.E + g.D + 1), cudaMemcpyHostToDevice, st);
+  // the array keeps the previous call's contents: counters start from zero every call
+  if (ce == cudaSuccess) ce = cudaMemsetAsync(d_hist, 0, sizeof(int32_t) * (size_t)kNaHistWords, st);
+  if (ce == cudaSuccess) ce = cudaMemsetAsync(d_gsize, 0, sizeof(int32_t) * (size_t)kNaGroupWords, st);
+  if (ce != cudaSuccess) return noalloc_fail(err, err_cap, EB_ERR_CUDA, cudaGetErrorString(ce));
+
+  const int gcap = EB_MAX_MB * (g.E + g.D * g.S);
+  const int chunk_blocks = (bp.n_chunks + kWarps - 1) / kWarps;
+  if (bp.n_chunks > 0) hist_kernel<<<chunk_blocks, kWarps * 32, 0, st>>>(mp, bp, d_res, topk_idx, d_hist);
+  sizes_kernel<<<(gcap + kWarps - 1) / kWarps, kWarps * 32, 0, st>>>(mp, bp, d_res, d_hist, d_cbase, d_gsize);
+  scan_kernel<<<1, 1024, 0, st>>>(mp, bp, d_res, d_gsize, group_off, group_w, step_meta);
+  if (bp.n_chunks > 0)
+    rank_kernel<<<chunk_blocks, kWarps * 32, 0, st>>>(mp, bp, d_res, topk_idx, d_cbase, group_off, pos, row_src);
+  if (bp.n_tok > 0)
+    gather_kernel<<<(bp.n_tok + kWarps - 1) / kWarps, kWarps * 32, 0, st>>>(bp.n_tok, g.H, g.K + g.S, (const uint4*)x,
+                                                                            pos, (uint4*)xp);
+  ce = cudaGetLastError();
+  if (ce != cudaSuccess) return noalloc_fail(err, err_cap, EB_ERR_CUDA, cudaGetErrorString(ce));
   return EB_OK;
 }
