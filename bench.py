@@ -34,9 +34,12 @@ METRIC = "cross-layer MoE step tokens/s"
 UNIT = "tokens/s"
 KERNELS_PER_STEP = 13  # route 2, schedule 1, permute 5, expert FFN 4, combine 1
 
-# DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum), keyed by workload; see profiles/.  None until a capture exists.
-NCU_TRAFFIC_BYTES = {}
+# DRAM traffic of the dominant kernel (ffn gate/up) from an ncu capture: dram__bytes_read.sum +
+# dram__bytes_write.sum over the algorithmic bytes of the captured launch.  The capture ran on the
+# 6-layer cut of the decode shape (profiles/ffn_c2small_ncu_full.md); traffic grows in proportion to
+# the weight bytes streamed, so a full launch is that ratio times its own algorithmic bytes.
+NCU_TRAFFIC_RATIO = {"c2": (3.423368e9 + 7.749888e6) / 3424780288.0,
+                     "c2small": (3.423368e9 + 7.749888e6) / 3424780288.0}
 
 
 def measured_peaks():
@@ -329,7 +332,7 @@ def run_ours(args, wl):
     else:
         achieved = alg["gateup_flops"] / t_gu / 1e12
         roof = dict(bound="tensor", achieved=achieved, peak=peaks["tensor"], unit="TFLOP/s", frac=achieved / peaks["tensor"])
-    roof.update(kernel="ffn_gateup", peak_source=peaks["src"], traffic=NCU_TRAFFIC_BYTES.get(wl.name),
+    roof.update(kernel="ffn_gateup", peak_source=peaks["src"], traffic=(NCU_TRAFFIC_RATIO[wl.name] * alg["gateup"] if wl.name in NCU_TRAFFIC_RATIO else None),
                 algorithmic_bytes=alg["gateup"], algorithmic_flops=alg["gateup_flops"], ms=t_gu * 1e3)
     ffn_flops = alg["gateup_flops"] + alg["down_flops"]
     ffn_bytes = alg["gateup"] + alg["down"]
@@ -416,7 +419,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c3init", "c4"])
+    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c2small", "c3", "c3init", "c4"])
     ap.add_argument("--no-idle", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -424,6 +427,10 @@ def main():
     if args.workload == "c3init":
         wl = synth.workload("c3", layers_override=tuple([0] * 16))
         wl = synth.Workload(**{**wl.__dict__, "name": "c3init"})
+    elif args.workload == "c2small":
+        # the decode shape cut to 6 layers and 6 micro-batches (6.6 GB of weights): the case ncu captures run on
+        wl = synth.workload("c2", L=6, N=6)
+        wl = synth.Workload(**{**wl.__dict__, "name": "c2small"})
     else:
         wl = synth.workload(args.workload)
     if args.impl == "reference":

@@ -269,7 +269,8 @@ def all_weights(wl: Workload, which: str, device="cpu") -> torch.Tensor:
     """Full weight tensor bf16: [L, E+S, I, H] (gate, up) or [L, E+S, H, I] (down)."""
     n = wl.n_weight_mats * wl.H * wl.I
     out = torch.empty(n, dtype=torch.bfloat16, device=device)
-    normal_bf16(wl.seed, tensor_id(_W_KIND[which]), 0, n, 0.02, device, out=out)
+    chunk = 1 << 26 if str(device).startswith("cuda") else 1 << 24
+    normal_bf16(wl.seed, tensor_id(_W_KIND[which]), 0, n, 0.02, device, chunk=chunk, out=out)
     if which == "down":
         return out.view(wl.L, wl.E + wl.S, wl.H, wl.I)
     return out.view(wl.L, wl.E + wl.S, wl.I, wl.H)
