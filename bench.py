@@ -225,6 +225,22 @@ def run_reference(args, wl):
     print(json.dumps(line))
 
 
+def replica_workload(wl, rank: int):
+    """Independent replicas: every rank draws its own batch, routing and weights."""
+    return synth.Workload(**{**wl.__dict__, "seed": wl.seed + rank}) if rank else wl
+
+
+def reduce_over_ranks(dist, device, ms: float, ms_e2e: float, tokens: float):
+    """Max over ranks of the two device times, sum over ranks of the tokens processed."""
+    if dist is None:
+        return ms, ms_e2e, tokens
+    v = torch.tensor([ms, ms_e2e], device=device, dtype=torch.float64)
+    dist.all_reduce(v, op=dist.ReduceOp.MAX)
+    tk = torch.tensor([tokens], device=device, dtype=torch.float64)
+    dist.all_reduce(tk, op=dist.ReduceOp.SUM)
+    return v[0].item(), v[1].item(), tk.item()
+
+
 def workload_config(wl):
     return dict(workload=f"{wl.name}: L={wl.L} E={wl.E} K={wl.K} S={wl.S} H={wl.H} I={wl.I} D={wl.D} "
                          f"map={wl.mapping} N={wl.N}x{wl.T} tokens at layers {wl.layers} m={wl.m} zipf_s={wl.zipf_s}",
@@ -244,8 +260,7 @@ def run_ours(args, wl):
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     torch.cuda.set_device(local)
     device = f"cuda:{local}"
-    if rank:  # independent replicas: every rank draws its own batch and routing
-        wl = synth.Workload(**{**wl.__dict__, "seed": wl.seed + rank})
+    wl = replica_workload(wl, rank)
     peaks = measured_peaks()
 
     step = B.from_workload(wl, device=device)
@@ -303,14 +318,7 @@ def run_ours(args, wl):
     barrier()
 
     # ---- reductions over ranks
-    tok_total, ms_max, ms_e2e_max = float(tokens_run), ms, ms_e2e
-    if dist is not None:
-        v = torch.tensor([ms, ms_e2e], device=device, dtype=torch.float64)
-        dist.all_reduce(v, op=dist.ReduceOp.MAX)
-        ms_max, ms_e2e_max = v.tolist()
-        tk = torch.tensor([tok_total], device=device, dtype=torch.float64)
-        dist.all_reduce(tk, op=dist.ReduceOp.SUM)
-        tok_total = tk.item()
+    ms_max, ms_e2e_max, tok_total = reduce_over_ranks(dist, device, ms, ms_e2e, float(tokens_run))
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()

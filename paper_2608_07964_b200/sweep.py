@@ -1,0 +1,81 @@
+"""Skew / micro-batch sweep on the 64-expert, top-6, hidden-2048 shape (8 layers, 8 virtual devices).
+
+    python -m paper_2608_07964_b200.sweep [--out results.md] [--policy 0]
+
+For every point (Zipf s, micro-batch count N, tokens per micro-batch T) it reports
+  * whole-run under-utilisation 1 - u of Algorithm 1 driven on the GPU (route + schedule every
+    step): cross-layer with m = ceil(0.75 N) and m = ceil(0.5 N), against every workload executed
+    alone and against lock-step execution (all micro-batches jointly, layer by layer);
+  * time and tokens/s of one full cross-layer step at the staggered state l_j = floor(j L / N).
+All arithmetic of the method runs in the library's kernels; this module only loops and prints.
+"""
+from __future__ import annotations
+
+import argparse
+import sys
+
+import torch
+
+from . import binding as B
+from . import driver, synth
+
+
+def timed_ms(fn, reps=5, warm=2):
+    for _ in range(warm):
+        fn()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record()
+    for _ in range(reps):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / reps
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--out", default=None)
+    ap.add_argument("--policy", type=int, default=B.POLICY_MAXUTIL)
+    ap.add_argument("--quick", action="store_true", help="s in {0, 1.0}, N in {4, 16} only")
+    args = ap.parse_args(argv)
+    dev = "cuda:0"
+    base = synth.workload_c5(2, 16, 0.0)
+    weights = tuple(synth.all_weights(base, k, dev) for k in ("gate", "up", "down"))
+    svals = [0.0, 1.0] if args.quick else [0.0, 0.5, 1.0, 1.5]
+    nvals = [4, 16] if args.quick else [2, 4, 8, 16]
+    lines = ["| s | N | T | steps EB(.75) | idle EB m=.75N | idle EB m=.5N | idle alone | idle lock-step | step ms | step tokens/s | step run/N |",
+             "|---|---|---|---|---|---|---|---|---|---|---|"]
+    for s in svals:
+        for N in nvals:
+            for T in (16, 128, 1024):
+                wl = synth.workload_c5(N, T, s)
+                bias = synth.zipf_bias(wl)
+                step = B.from_workload(wl, device=dev)
+                step.bind_weights(*weights)
+                logits_of = lambda j, l: synth.logits_for(wl, j, l, dev, bias)
+                m75, m50 = wl.m, -(-N // 2)
+                tr75 = driver.run_load_trace(step, wl.tok_off, wl.L, m75, args.policy, logits_of)
+                tr50 = driver.run_load_trace(step, wl.tok_off, wl.L, m50, args.policy, logits_of)
+                lock = driver.run_load_trace(step, wl.tok_off, wl.L, N, B.POLICY_ALL, logits_of)
+                f75, f50, fl = (driver.idle_fractions(t, wl.D) for t in (tr75, tr50, lock))
+                # one full step at the staggered state
+                step.logits[:wl.T_tot].copy_(synth.packed_logits(wl, device=dev))
+                step.x[:wl.T_tot].copy_(synth.packed_hidden(wl, device=dev))
+                batch = B.Batch(wl.tok_off, wl.layers)
+                ms = timed_ms(lambda: step.eb_step(batch, m75, args.policy))
+                run = step.sched_result()["n_run"]
+                assert step.device_status() == 0
+                lines.append(f"| {s} | {N} | {T} | {f75['steps']} | {f75['idle_cross_layer']:.3f} | {f50['idle_cross_layer']:.3f} | "
+                             f"{f75['idle_each_alone']:.3f} | {fl['idle_cross_layer']:.3f} | {ms:.3f} | {run * T / ms * 1e3:.0f} | {run}/{N} |")
+                step.close()
+                print(lines[-1], flush=True)
+    text = "\n".join(lines) + "\n"
+    if args.out:
+        with open(args.out, "w") as f:
+            f.write(text)
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
