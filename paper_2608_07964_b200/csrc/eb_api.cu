@@ -68,13 +68,19 @@ static size_t carve(eb_ctx* c, char* base) {
   c->max_mtiles = rows / 128 + gcap;
   c->max_work1 = c->max_mtiles * ((g.I + 127) / 128);
   c->max_work2 = c->max_mtiles * ((g.H + 255) / 256);
+  const int max_ptiles = rows / 256 + gcap;
+  c->max_work1p = max_ptiles * ((g.I + 127) / 128);
+  c->max_work2p = max_ptiles * ((g.H + 255) / 256);
   c->chunk_hist = (int32_t*)take(sizeof(int32_t) * (size_t)c->max_chunks * g.E);
   c->chunk_base = (int32_t*)take(sizeof(int32_t) * (size_t)c->max_chunks * g.E);
   c->group_size = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
   c->mtile_pref = (int32_t*)take(sizeof(int32_t) * (size_t)(gcap + 1));
-  c->work_count = (int32_t*)take(sizeof(int32_t) * 4);
+  c->ptile_pref = (int32_t*)take(sizeof(int32_t) * (size_t)(gcap + 1));
+  c->work_count = (int32_t*)take(sizeof(int32_t) * 8);
   c->work1 = (int4*)take(sizeof(int4) * (size_t)c->max_work1);
   c->work2 = (int4*)take(sizeof(int4) * (size_t)c->max_work2);
+  c->work1p = (int4*)take(sizeof(int4) * (size_t)c->max_work1p);
+  c->work2p = (int4*)take(sizeof(int4) * (size_t)c->max_work2p);
   c->act = (bf16*)take(sizeof(bf16) * (size_t)rows * g.I);
   return off;
 }
@@ -254,7 +260,7 @@ extern "C" eb_status eb_device_status(eb_ctx* c, int32_t* out_status) {
 
 static const char* kKernelNames[EBK_COUNT] = {
     "route", "schedule", "permute_hist", "permute_sizes", "permute_scan", "permute_rank",
-    "permute_gather", "ffn_plan", "ffn_fill", "ffn_gateup", "ffn_down", "combine"};
+    "permute_gather", "ffn_plan", "ffn_fill", "ffn_gateup", "ffn_down", "ffn_gateup_pair", "ffn_down_pair", "combine"};
 
 extern "C" int32_t eb_num_kernels(void) { return EBK_COUNT; }
 extern "C" const char* eb_kernel_name(int32_t i) { return (i >= 0 && i < EBK_COUNT) ? kKernelNames[i] : ""; }

@@ -18,6 +18,13 @@
 // the extra rows are never stored), which keeps shared-memory fill traffic close to the weight
 // bytes in the weight-streaming regime.
 //
+// Groups with many rows run on CTA pairs instead (ffn_kernel<PHASE, true>, a 2-CTA cluster): the pair
+// owns a 256-row tile, each CTA loads its own 128 rows of A and one half of the weight tile (for
+// gate/up: CTA 0 the gate rows, CTA 1 the up rows), and the leader CTA issues tcgen05.mma
+// cta_group::2 (M = 256) that reads both halves.  A stage shrinks from 48 KB to 32 KB per CTA for the
+// same tensor-core time, so the ring deepens to 6 stages and L2 traffic per flop drops by a third -
+// that is what the tensor-bound regime needs.  No load is multicast; only tcgen05.commit is.
+//
 // Every wait on an mbarrier is bounded: on expiry the kernel records EB_ERR_TIMEOUT in the
 // context status word, lets copies in flight land, frees its TMEM and returns.
 #include "eb_internal.cuh"
@@ -33,9 +40,12 @@ constexpr int kABytes = BM * BK * 2;
 constexpr int kASmallBytes = kSmallRows * BK * 2;
 constexpr int kBBytes = BN * BK * 2;
 constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kPairStages = 6;
+constexpr int kPairStageBytes = kABytes + kBBytes / 2;   // per CTA of a pair: own A rows + half of B
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 512;
 constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+static_assert(kPairStages * kPairStageBytes == kStages * kStageBytes, "both variants use the same ring size");
 constexpr long long kSpinLimitCycles = 4000000000LL;
 
 // ---- PTX wrappers ----------------------------------------------------------------------------
@@ -94,6 +104,62 @@ __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
 
+// ---- CTA-pair (cta_group::2) forms ------------------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA loads whose completion is counted on a barrier that may live in the peer CTA (never multicast)
+__device__ __forceinline__ void tma_pair_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_pair_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B^T with M = 256 (128 rows per CTA), N = 256, K = 16
+__device__ __forceinline__ void umma_pair_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+// arrives on the barrier at this offset in both CTAs of the pair once the MMAs issued so far are done
+__device__ __forceinline__ void umma_pair_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3)
+               : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -137,6 +203,8 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 }
 // Instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = 256, M = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+// Same with M = 256 for the CTA-pair instruction.
+constexpr uint32_t kIdescPair = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
@@ -144,80 +212,101 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 }
 __device__ __forceinline__ float silu_mul(uint32_t g_bits, uint32_t u_bits) {
   float g = __uint_as_float(g_bits), u = __uint_as_float(u_bits);
-  return g / (1.0f + __expf(-g)) * u;
+  return __fdividef(g, 1.0f + __expf(-g)) * u;
 }
 
 // ---- the grouped GEMM kernel -----------------------------------------------------------------
-// PHASE 1: gate/up + SwiGLU (output tile 128 x 128);  PHASE 2: down (output tile 128 x 256).
-template <int PHASE>
+// PHASE 1: gate/up + SwiGLU (output 128 columns per tile);  PHASE 2: down (output 256 columns per tile).
+// PAIR false: one CTA per 128-row tile.  PAIR true: a 2-CTA cluster per 256-row tile.
+template <int PHASE, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA_small,
            const __grid_constant__ CUtensorMap tmB0, const __grid_constant__ CUtensorMap tmB1,
            const int4* __restrict__ work, const int32_t* __restrict__ work_count, bf16* __restrict__ out,
            int ld_out, int n_out, int k_total, int* status) {
+  constexpr int NS = PAIR ? kPairStages : kStages;
+  constexpr int SB = PAIR ? kPairStageBytes : kStageBytes;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - raw);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStages * kStageBytes);
-  // barrier indices: full[0..S), empty[S..2S), tmem_full[2S, 2S+2), tmem_empty[2S+2, 2S+4)
-  const uint32_t bar0 = base + kStages * kStageBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)NS * SB);
+  // barrier indices: full[0..NS), empty[NS..2NS), tmem_full[2NS, 2NS+2), tmem_empty[2NS+2, 2NS+4)
+  const uint32_t bar0 = base + NS * SB;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
-  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + a); };
-  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 + a); };
-  volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(bars + 2 * kStages + 4);
-  volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 2 * kStages + 5);
+  auto empty_bar = [&](int s) { return bar0 + 8u * (NS + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * NS + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * NS + 2 + a); };
+  volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(bars + 2 * NS + 4);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 2 * NS + 5);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;   // CTA 0 of a pair is the leader
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(full_bar(s), 1);
-      mbar_init(empty_bar(s), 1);
+    for (int s = 0; s < NS; ++s) {
+      mbar_init(full_bar(s), 1);    // producer's arrive + all bytes of the stage (pair: of both CTAs, leader only)
+      mbar_init(empty_bar(s), 1);   // one tcgen05.commit
     }
     for (int a = 0; a < 2; ++a) {
-      mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), 4);
+      mbar_init(tfull_bar(a), 1);                // one tcgen05.commit
+      mbar_init(tempty_bar(a), PAIR ? 8 : 4);    // one arrival per epilogue warp (pair: of both CTAs, leader only)
     }
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     prefetch_tmap(&tmA);
-    prefetch_tmap(&tmA_small);
+    if (!PAIR) prefetch_tmap(&tmA_small);
     prefetch_tmap(&tmB0);
     if (PHASE == 1) prefetch_tmap(&tmB1);
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32((const void*)s_tmem), kTmemCols);
-    tmem_relinquish();
+    if (PAIR) {
+      tmem_alloc_pair(smem_u32((const void*)s_tmem), kTmemCols);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(smem_u32((const void*)s_tmem), kTmemCols);
+      tmem_relinquish();
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();   // the peer's barriers are initialised before anything arrives on them
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
-  const int n_work = work_count[PHASE - 1];
+  const int n_work = work_count[(PAIR ? 5 : 0) + PHASE - 1];
   const int num_kb = (k_total + BK - 1) / BK;
+  const int w_first = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int w_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
-      for (int w = blockIdx.x; w < n_work; w += gridDim.x) {
+      for (int w = w_first; w < n_work; w += w_step) {
         const int4 it = __ldg(work + w);  // x = first row, y = valid rows, z = weight matrix, w = n tile
-        const bool small = it.y <= kSmallRows;
-        const uint32_t tx = (small ? kASmallBytes : kABytes) + kBBytes;
+        const bool small = !PAIR && it.y <= kSmallRows;
+        const uint32_t tx = PAIR ? 2u * kPairStageBytes : (uint32_t)((small ? kASmallBytes : kABytes) + kBBytes);
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, s_abort, status)) goto done;
-          const uint32_t sa = base + stage * kStageBytes, sb = sa + kABytes;
-          mbar_expect_tx(full_bar(stage), tx);
-          tma_load_2d(sa, small ? &tmA_small : &tmA, kb * BK, it.x, full_bar(stage));
-          if (PHASE == 1) {
-            tma_load_3d(sb, &tmB0, kb * BK, it.w * 128, it.z, full_bar(stage));
-            tma_load_3d(sb + kBBytes / 2, &tmB1, kb * BK, it.w * 128, it.z, full_bar(stage));
+          const uint32_t sa = base + stage * SB, sb = sa + kABytes;
+          if (PAIR) {
+            // both CTAs' copies are counted on the leader's barrier; the leader announces the total
+            const uint32_t fb = map_to_cta(full_bar(stage), 0);
+            if (rank == 0) mbar_expect_tx(full_bar(stage), tx);
+            tma_pair_load_2d(sa, &tmA, kb * BK, it.x + (int)rank * BM, fb);
+            if (PHASE == 1) tma_pair_load_3d(sb, rank == 0 ? &tmB0 : &tmB1, kb * BK, it.w * 128, it.z, fb);
+            else tma_pair_load_3d(sb, &tmB0, kb * BK, it.w * BN + (int)rank * 128, it.z, fb);
           } else {
-            tma_load_3d(sb, &tmB0, kb * BK, it.w * BN, it.z, full_bar(stage));
+            mbar_expect_tx(full_bar(stage), tx);
+            tma_load_2d(sa, small ? &tmA_small : &tmA, kb * BK, it.x, full_bar(stage));
+            if (PHASE == 1) {
+              tma_load_3d(sb, &tmB0, kb * BK, it.w * 128, it.z, full_bar(stage));
+              tma_load_3d(sb + kBBytes / 2, &tmB1, kb * BK, it.w * 128, it.z, full_bar(stage));
+            } else {
+              tma_load_3d(sb, &tmB0, kb * BK, it.w * BN, it.z, full_bar(stage));
+            }
           }
-          if (++stage == kStages) {
+          if (++stage == NS) {
             stage = 0;
             phase ^= 1u;
           }
@@ -225,12 +314,12 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
-    if (lane == 0) {
+    // ---------------- MMA issuer (pair: leader CTA only) ----------------
+    if (lane == 0 && rank == 0) {
       int stage = 0;
       uint32_t phase = 0;
       int local = 0;
-      for (int w = blockIdx.x; w < n_work; w += gridDim.x, ++local) {
+      for (int w = w_first; w < n_work; w += w_step, ++local) {
         const int as = local & 1;
         const uint32_t aphase = (local >> 1) & 1u;
         if (!mbar_wait(tempty_bar(as), aphase ^ 1u, s_abort, status)) goto done;
@@ -239,31 +328,35 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, s_abort, status)) goto done;
           tc_fence_after();
-          const uint32_t sa = base + stage * kStageBytes, sb = sa + kABytes;
+          const uint32_t sa = base + stage * SB, sb = sa + kABytes;
           const uint64_t da = smem_desc(sa), db = smem_desc(sb);
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k)
-            umma_bf16(d_tmem, da + 2 * k, db + 2 * k, kIdesc, (kb | k) != 0 ? 1u : 0u);
-          umma_commit(empty_bar(stage));  // smem stage reusable once these MMAs have read it
-          if (++stage == kStages) {
+          for (int k = 0; k < BK / 16; ++k) {
+            if (PAIR) umma_pair_bf16(d_tmem, da + 2 * k, db + 2 * k, kIdescPair, (kb | k) != 0 ? 1u : 0u);
+            else umma_bf16(d_tmem, da + 2 * k, db + 2 * k, kIdesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          // smem stage reusable (in both CTAs of a pair) once these MMAs have read it
+          if (PAIR) umma_pair_commit(empty_bar(stage)); else umma_commit(empty_bar(stage));
+          if (++stage == NS) {
             stage = 0;
             phase ^= 1u;
           }
         }
-        umma_commit(tfull_bar(as));  // accumulator complete
+        // accumulator complete
+        if (PAIR) umma_pair_commit(tfull_bar(as)); else umma_commit(tfull_bar(as));
       }
     }
   } else {
     // ---------------- epilogue warps ----------------
     const int q = warp & 3;  // TMEM lane quadrant this warp may read
     int local = 0;
-    for (int w = blockIdx.x; w < n_work; w += gridDim.x, ++local) {
+    for (int w = w_first; w < n_work; w += w_step, ++local) {
       const int4 it = __ldg(work + w);
       const int as = local & 1;
       const uint32_t aphase = (local >> 1) & 1u;
       if (!mbar_wait(tfull_bar(as), aphase, s_abort, status)) goto done;
       tc_fence_after();
-      const int r = q * 32 + lane;
+      const int r = (int)rank * BM + q * 32 + lane;   // row inside the (pair's) tile
       const bool row_ok = r < it.y;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + as * BN;
       if (PHASE == 1) {
@@ -321,7 +414,10 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
       // all TMEM reads of this warp are complete (wait::ld above): hand the accumulator back
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(as));
+      if (lane == 0) {
+        if (PAIR) mbar_arrive_cluster(map_to_cta(tempty_bar(as), 0));
+        else mbar_arrive(tempty_bar(as));
+      }
     }
   }
 
@@ -332,19 +428,30 @@ done:
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();   // neither CTA leaves while its peer may still touch its memory or barriers
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, kTmemCols);
+    if (PAIR) tmem_dealloc_pair(tmem_base, kTmemCols); else tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
 // ---- tile list construction ------------------------------------------------------------------
-// plan: per group of the requested range, number of 128-row tiles; exclusive scan; totals.
+// A group runs either on single CTAs (128-row tiles) or on CTA pairs (256-row tiles), never both, so
+// its weights are streamed by one kernel only.  Pairs are used when they do not add padded rows
+// compared with 128-row tiles, or when the group is large enough for the padding not to matter.
+__device__ __forceinline__ bool group_uses_pairs(int rows) {
+  const int rem = rows % (2 * BM);
+  return rows > BM && (rows >= 4 * BM || rem == 0 || rem > BM);
+}
+
+// plan: per group of the requested range, number of 128-row tiles or of 256-row pair tiles;
+// exclusive scans of both; totals.
 __global__ void __launch_bounds__(1024)
 plan_kernel(const int32_t* __restrict__ group_off, const int32_t* __restrict__ step_meta, int device, int nt1, int nt2,
-            int32_t* __restrict__ mtile_pref, int32_t* __restrict__ work_count) {
-  __shared__ int s_warp[32];
-  __shared__ int s_carry;
+            int allow_pairs, int32_t* __restrict__ mtile_pref, int32_t* __restrict__ ptile_pref,
+            int32_t* __restrict__ work_count) {
+  __shared__ long long s_warp[32];
+  __shared__ long long s_carry;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = step_meta[1];
   const int g0 = device < 0 ? 0 : step_meta[3 + device];
@@ -354,77 +461,93 @@ plan_kernel(const int32_t* __restrict__ group_off, const int32_t* __restrict__ s
   __syncthreads();
   for (int b = 0; b < ng; b += 1024) {
     int i = b + tid;
-    int v = 0;
-    if (i < ng) v = (group_off[g0 + i + 1] - group_off[g0 + i] + BM - 1) / BM;
-    int incl = v;
+    long long v = 0;  // low 32 bits: single tiles, high 32 bits: pair tiles
+    if (i < ng) {
+      int rows = group_off[g0 + i + 1] - group_off[g0 + i];
+      if (allow_pairs && group_uses_pairs(rows)) v = (long long)((rows + 2 * BM - 1) / (2 * BM)) << 32;
+      else v = (rows + BM - 1) / BM;
+    }
+    long long incl = v;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      int n = __shfl_up_sync(0xffffffffu, incl, o);
+      long long n = __shfl_up_sync(0xffffffffu, incl, o);
       if (lane >= o) incl += n;
     }
     if (lane == 31) s_warp[warp] = incl;
     __syncthreads();
     if (warp == 0) {
-      int wv = s_warp[lane], wi = wv;
+      long long wv = s_warp[lane], wi = wv;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
-        int n = __shfl_up_sync(0xffffffffu, wi, o);
+        long long n = __shfl_up_sync(0xffffffffu, wi, o);
         if (lane >= o) wi += n;
       }
       s_warp[lane] = wi - wv;
     }
     __syncthreads();
-    int excl = s_carry + s_warp[warp] + incl - v;
-    if (i < ng) mtile_pref[i] = excl;
+    long long excl = s_carry + s_warp[warp] + incl - v;
+    if (i < ng) {
+      mtile_pref[i] = (int)(excl & 0xffffffffLL);
+      ptile_pref[i] = (int)(excl >> 32);
+    }
     __syncthreads();
     if (tid == 1023) s_carry = excl + v;
     __syncthreads();
   }
   if (tid == 0) {
-    int mt = s_carry;
+    const int mt = (int)(s_carry & 0xffffffffLL), pt = (int)(s_carry >> 32);
     mtile_pref[ng] = mt;
+    ptile_pref[ng] = pt;
     work_count[0] = mt * nt1;
     work_count[1] = mt * nt2;
     work_count[2] = mt;
     work_count[3] = g0;
     work_count[4] = ng;
+    work_count[5] = pt * nt1;
+    work_count[6] = pt * nt2;
+    work_count[7] = pt;
   }
 }
 
-// fill: one thread per tile; tiles of a group are ordered n-tile major, m-tile minor.
+// fill: one thread per tile of the four lists (single gate/up, single down, pair gate/up, pair down);
+// tiles of a group are ordered weight-tile major, row-tile minor.
 __global__ void __launch_bounds__(256)
 fill_kernel(const int32_t* __restrict__ group_off, const int32_t* __restrict__ group_w,
-            const int32_t* __restrict__ mtile_pref, const int32_t* __restrict__ work_count, int nt1, int nt2,
-            int max1, int max2, int4* __restrict__ work1, int4* __restrict__ work2) {
-  const int w1 = work_count[0], w2 = work_count[1], g0 = work_count[3], ng = work_count[4];
-  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < w1 + w2; idx += gridDim.x * blockDim.x) {
-    const bool first = idx < w1;
-    const int local = first ? idx : idx - w1;
-    const int nt = first ? nt1 : nt2;
-    const int mt_index = local / nt;  // position in units of "m-tiles x nt": find group by m-tile prefix
-    // largest gi with mtile_pref[gi] * nt <= local  <=>  mtile_pref[gi] <= local / nt
+            const int32_t* __restrict__ mtile_pref, const int32_t* __restrict__ ptile_pref,
+            const int32_t* __restrict__ work_count, int nt1, int nt2, int max1, int max2, int maxp1, int maxp2,
+            int4* __restrict__ work1, int4* __restrict__ work2, int4* __restrict__ work1p, int4* __restrict__ work2p) {
+  const int g0 = work_count[3], ng = work_count[4];
+  const int cnt[4] = {work_count[0], work_count[1], work_count[5], work_count[6]};
+  const int total = cnt[0] + cnt[1] + cnt[2] + cnt[3];
+  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+    int list = 0, local = idx;
+    while (local >= cnt[list]) local -= cnt[list++];
+    const bool pair = list >= 2;
+    const int nt = (list & 1) ? nt2 : nt1;
+    const int tile_rows = pair ? 2 * BM : BM;
+    const int32_t* pref = pair ? ptile_pref : mtile_pref;
+    const int t_index = local / nt;
+    // largest gi with pref[gi] <= t_index: groups without tiles in this list share their successor's
+    // prefix, and a group that owns tiles has pref[gi + 1] > pref[gi]
     int lo = 0, hi = ng - 1;
     while (lo < hi) {
       int mid = (lo + hi + 1) >> 1;
-      if (mtile_pref[mid] <= mt_index) lo = mid; else hi = mid - 1;
+      if (pref[mid] <= t_index) lo = mid; else hi = mid - 1;
     }
-    // skip past empty groups that share the same prefix value: take the last group with that prefix
     const int gi = lo;
-    const int mt_g = mtile_pref[gi + 1] - mtile_pref[gi];
-    const int rem = local - mtile_pref[gi] * nt;
-    const int n = rem / mt_g, m = rem % mt_g;
+    const int t_g = pref[gi + 1] - pref[gi];
+    const int rem = local - pref[gi] * nt;
+    const int n = rem / t_g, m = rem % t_g;
     const int g = g0 + gi;
-    const int row0 = group_off[g] + m * BM;
+    const int row0 = group_off[g] + m * tile_rows;
     int4 it;
     it.x = row0;
-    it.y = min(BM, group_off[g + 1] - row0);
+    it.y = min(tile_rows, group_off[g + 1] - row0);
     it.z = group_w[g];
     it.w = n;
-    if (first) {
-      if (local < max1) work1[local] = it;
-    } else {
-      if (local < max2) work2[local] = it;
-    }
+    int4* dst = list == 0 ? work1 : list == 1 ? work2 : list == 2 ? work1p : work2p;
+    const int cap = list == 0 ? max1 : list == 1 ? max2 : list == 2 ? maxp1 : maxp2;
+    if (local < cap) dst[local] = it;
   }
 }
 
@@ -460,6 +583,26 @@ bool make_map(CUtensorMap* m, const void* ptr, uint64_t d0, uint64_t d1, uint64_
   return r == CUDA_SUCCESS;
 }
 
+template <int PHASE, bool PAIR>
+cudaError_t launch_ffn(eb_ctx* c, cudaStream_t st, const CUtensorMap& tA, const CUtensorMap& tAs, const CUtensorMap& tB0,
+                       const CUtensorMap& tB1, const int4* work, bf16* out, int ld_out, int n_out, int k_total) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(PAIR ? c->pair_grid : c->num_sms);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const int32_t* wc = c->work_count;
+  return cudaLaunchKernelEx(&cfg, ffn_kernel<PHASE, PAIR>, tA, tAs, tB0, tB1, work, wc, out, ld_out, n_out, k_total,
+                            c->d_status);
+}
+
 }  // namespace
 
 eb_status ebi_ffn_bind(eb_ctx* c) {
@@ -467,15 +610,39 @@ eb_status ebi_ffn_bind(eb_ctx* c) {
   const uint64_t nw = (uint64_t)g.L * (g.E + g.S);
   if (!make_map(&c->tm_gate, c->w_gate, g.H, g.I, nw, BK, 128) ||
       !make_map(&c->tm_up, c->w_up, g.H, g.I, nw, BK, 128) ||
-      !make_map(&c->tm_down, c->w_down, g.I, g.H, nw, BK, BN))
+      !make_map(&c->tm_down, c->w_down, g.I, g.H, nw, BK, BN) ||
+      !make_map(&c->tm_down_half, c->w_down, g.I, g.H, nw, BK, 128))
     return ebi_fail(c, EB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the weights");
   static bool attr_set = false;
+  static int pair_grid = 0;
   if (!attr_set) {
-    cudaError_t e1 = cudaFuncSetAttribute(ffn_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    cudaError_t e2 = cudaFuncSetAttribute(ffn_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e1 != cudaSuccess || e2 != cudaSuccess) return ebi_check_cuda(c, e1 != cudaSuccess ? e1 : e2, "cudaFuncSetAttribute");
+    cudaError_t e = cudaFuncSetAttribute(ffn_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e != cudaSuccess) return ebi_check_cuda(c, e, "cudaFuncSetAttribute");
+    // how many 2-CTA clusters of this kernel the device can hold at once (one CTA per SM)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * (c->num_sms / 2));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    e = cudaOccupancyMaxActiveClusters(&clusters, ffn_kernel<1, true>, &cfg);
+    if (e != cudaSuccess || clusters < 1) {
+      cudaGetLastError();
+      clusters = 0;   // pairs unavailable: every group runs on single CTAs
+    }
+    pair_grid = 2 * (clusters < c->num_sms / 2 ? clusters : c->num_sms / 2);
     attr_set = true;
   }
+  c->pair_grid = pair_grid;
   return EB_OK;
 }
 
@@ -492,25 +659,36 @@ eb_status ebi_ffn_run(eb_ctx* c, cudaStream_t st, const void* xp, const int32_t*
       !make_map(&tm_a, c->act, g.I, rows, 0, BK, BM) || !make_map(&tm_as, c->act, g.I, rows, 0, BK, kSmallRows))
     return ebi_fail(c, EB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the activations");
   const int nt1 = (g.I + 127) / 128, nt2 = (g.H + BN - 1) / BN;
+  const bool pairs = c->pair_grid >= 2 && c->cfg.max_tokens > BM;   // no group can exceed 128 rows otherwise
   {
     KernelTimer timer(c, EBK_FFN_PLAN, st);
-    plan_kernel<<<1, 1024, 0, st>>>(group_off, step_meta, device, nt1, nt2, c->mtile_pref, c->work_count);
+    plan_kernel<<<1, 1024, 0, st>>>(group_off, step_meta, device, nt1, nt2, pairs ? 1 : 0, c->mtile_pref, c->ptile_pref,
+                                    c->work_count);
   }
   {
     KernelTimer timer(c, EBK_FFN_FILL, st);
-    fill_kernel<<<c->num_sms, 256, 0, st>>>(group_off, group_w, c->mtile_pref, c->work_count, nt1, nt2, c->max_work1,
-                                            c->max_work2, c->work1, c->work2);
+    fill_kernel<<<c->num_sms, 256, 0, st>>>(group_off, group_w, c->mtile_pref, c->ptile_pref, c->work_count, nt1, nt2,
+                                            c->max_work1, c->max_work2, c->max_work1p, c->max_work2p, c->work1, c->work2,
+                                            c->work1p, c->work2p);
   }
-  {
+  cudaError_t e = cudaSuccess;
+  if (pairs) {
+    KernelTimer timer(c, EBK_FFN_GATEUP_PAIR, st);
+    e = launch_ffn<1, true>(c, st, tm_x, tm_xs, c->tm_gate, c->tm_up, c->work1p, c->act, g.I, g.I, g.H);
+  }
+  if (e == cudaSuccess) {
     KernelTimer timer(c, EBK_FFN_GATEUP, st);
-    ffn_kernel<1><<<c->num_sms, kThreads, kSmemBytes, st>>>(tm_x, tm_xs, c->tm_gate, c->tm_up, c->work1, c->work_count,
-                                                            c->act, g.I, g.I, g.H, c->d_status);
+    e = launch_ffn<1, false>(c, st, tm_x, tm_xs, c->tm_gate, c->tm_up, c->work1, c->act, g.I, g.I, g.H);
   }
-  {
+  if (e == cudaSuccess && pairs) {
+    KernelTimer timer(c, EBK_FFN_DOWN_PAIR, st);
+    e = launch_ffn<2, true>(c, st, tm_a, tm_as, c->tm_down_half, c->tm_down_half, c->work2p, (bf16*)yp, g.H, g.H, g.I);
+  }
+  if (e == cudaSuccess) {
     KernelTimer timer(c, EBK_FFN_DOWN, st);
-    ffn_kernel<2><<<c->num_sms, kThreads, kSmemBytes, st>>>(tm_a, tm_as, c->tm_down, c->tm_down, c->work2, c->work_count,
-                                                            (bf16*)yp, g.H, g.H, g.I, c->d_status);
+    e = launch_ffn<2, false>(c, st, tm_a, tm_as, c->tm_down, c->tm_down, c->work2, (bf16*)yp, g.H, g.H, g.I);
   }
+  if (e != cudaSuccess) return ebi_check_cuda(c, e, "expert_ffn launch");
   EB_LAUNCH_CHECK(c, "expert_ffn");
   return EB_OK;
 }

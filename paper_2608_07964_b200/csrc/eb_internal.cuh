@@ -26,6 +26,8 @@ enum EbKernel {
   EBK_FFN_FILL,
   EBK_FFN_GATEUP,
   EBK_FFN_DOWN,
+  EBK_FFN_GATEUP_PAIR,
+  EBK_FFN_DOWN_PAIR,
   EBK_COMBINE,
   EBK_COUNT
 };
@@ -61,7 +63,8 @@ struct eb_ctx {
   const bf16* w_gate = nullptr;
   const bf16* w_up = nullptr;
   const bf16* w_down = nullptr;
-  CUtensorMap tm_gate, tm_up, tm_down;
+  CUtensorMap tm_gate, tm_up, tm_down, tm_down_half;
+  int pair_grid = 0;               // CTAs launched for the CTA-pair kernels (0: pairs unavailable)
 
   // workspace carve-up
   void* ws = nullptr;
@@ -69,12 +72,15 @@ struct eb_ctx {
   int32_t* chunk_hist = nullptr;   // [max_chunks][E]
   int32_t* chunk_base = nullptr;   // [max_chunks][E]
   int32_t* group_size = nullptr;   // [G_cap]
-  int32_t* mtile_pref = nullptr;   // [G_cap + 1]
-  int32_t* work_count = nullptr;   // [4]: gate/up items, down items, m-tiles
+  int32_t* mtile_pref = nullptr;   // [G_cap + 1] 128-row tiles before each group
+  int32_t* ptile_pref = nullptr;   // [G_cap + 1] 256-row pair tiles before each group
+  int32_t* work_count = nullptr;   // [8]: tile counts of the four lists, group range
   int4* work1 = nullptr;           // gate/up tile list
   int4* work2 = nullptr;           // down tile list
+  int4* work1p = nullptr;          // gate/up tile list of the CTA-pair kernel
+  int4* work2p = nullptr;          // down tile list of the CTA-pair kernel
   bf16* act = nullptr;             // [R_cap][I]
-  int32_t max_chunks = 0, max_mtiles = 0, max_work1 = 0, max_work2 = 0;
+  int32_t max_chunks = 0, max_mtiles = 0, max_work1 = 0, max_work2 = 0, max_work1p = 0, max_work2p = 0;
 
   bool timing = false;
   cudaEvent_t ev[2 * EBK_COUNT] = {};

@@ -302,3 +302,25 @@ def test_argument_errors_return_codes():
         step.eb_expert_ffn_grouped()                 # weights not bound
     assert e.value.code == 1
     assert step.device_status() == 0
+
+
+# ----------------------------------------------------------------------------------- CTA-pair tiles
+def test_group_sizes_around_the_pair_tile_boundaries():
+    """Exact group sizes on both sides of every rule that sends a group to 128-row tiles on single CTAs
+    or to 256-row tiles on CTA pairs; every row of every group is compared."""
+    B = _binding()
+    sizes = [129, 256, 257, 384, 385, 512, 513, 640, 100, 1, 128, 0, 300, 768]
+    E = len(sizes)
+    wl = synth.Workload(name="pairs", L=1, E=E, K=1, S=0, H=192, I=328, D=2, mapping="mod", N=1, T=sum(sizes),
+                        zipf_s=0.0)
+    store = Hn.WeightStore(wl)
+    case = Hn.make_case(wl)
+    logits = torch.full((wl.T, E), -4.0)
+    t = 0
+    for e, n in enumerate(sizes):
+        logits[t:t + n, e] = 6.0
+        t += n
+    perm = torch.from_numpy(np.random.default_rng(5).permutation(wl.T))
+    case.logits = logits[perm].contiguous()
+    step, ref = _full_step(case, store, 1)
+    assert sorted(np.diff(ref["group_off"]).tolist()) == sorted(sizes)
