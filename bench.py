@@ -38,8 +38,8 @@ KERNELS_PER_STEP = 15  # route 2, schedule 1, permute 5, expert FFN 6 (plan, fil
 # dram__bytes_write.sum over the algorithmic bytes of the captured launch.  The capture ran on the
 # 6-layer cut of the decode shape (profiles/ffn_c2small_ncu_full.md); traffic grows in proportion to
 # the weight bytes streamed, so a full launch is that ratio times its own algorithmic bytes.
-NCU_TRAFFIC_RATIO = {"c2": (3.423368e9 + 7.749888e6) / 3424780288.0,
-                     "c2small": (3.423368e9 + 7.749888e6) / 3424780288.0}
+NCU_TRAFFIC_RATIO = {"c2": (3.421758e9 + 8.032256e6) / 3424780288.0,
+                     "c2small": (3.421758e9 + 8.032256e6) / 3424780288.0}
 
 
 def measured_peaks():

@@ -659,7 +659,10 @@ eb_status ebi_ffn_run(eb_ctx* c, cudaStream_t st, const void* xp, const int32_t*
       !make_map(&tm_a, c->act, g.I, rows, 0, BK, BM) || !make_map(&tm_as, c->act, g.I, rows, 0, BK, kSmallRows))
     return ebi_fail(c, EB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the activations");
   const int nt1 = (g.I + 127) / 128, nt2 = (g.H + BN - 1) / BN;
-  const bool pairs = c->pair_grid >= 2 && c->cfg.max_tokens > BM;   // no group can exceed 128 rows otherwise
+  // CTA pairs only pay for groups of more than 128 rows; skip their launches when the permutation that
+  // produced this step (same step_meta buffer) says no group can be that large
+  bool pairs = c->pair_grid >= 2 && c->cfg.max_tokens > BM;
+  if (pairs && c->hint_meta == step_meta && c->hint_max_group_rows >= 0 && c->hint_max_group_rows <= BM) pairs = false;
   {
     KernelTimer timer(c, EBK_FFN_PLAN, st);
     plan_kernel<<<1, 1024, 0, st>>>(group_off, step_meta, device, nt1, nt2, pairs ? 1 : 0, c->mtile_pref, c->ptile_pref,

@@ -65,6 +65,10 @@ struct eb_ctx {
   const bf16* w_down = nullptr;
   CUtensorMap tm_gate, tm_up, tm_down, tm_down_half;
   int pair_grid = 0;               // CTAs launched for the CTA-pair kernels (0: pairs unavailable)
+  // Host-side hint left by the last eb_permute: the largest number of tokens sitting at one layer,
+  // an upper bound on the rows of any group of that step, and the step_meta buffer it belongs to.
+  int32_t hint_max_group_rows = -1;
+  const int32_t* hint_meta = nullptr;
 
   // workspace carve-up
   void* ws = nullptr;
