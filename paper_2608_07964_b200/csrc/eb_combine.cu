@@ -1,14 +1,15 @@
 // eb_combine: weighted aggregation of Eq. 1 in gather form.
 //
-// One warp per token.  For every 16-byte column vector the warp loads the K + S expert-output
-// rows of the token (independent loads, all in flight together), accumulates in fp32 in the
+// A team of threads per token, one 16-byte column vector each (a whole row in flight at once).  A
+// thread loads its vector from the K + S expert-output rows of the token (independent loads, all
+// in flight together), accumulates in fp32 in the
 // fixed order k = 0..K-1 then s = 0..S-1, and stores bf16 (round to nearest even).  Gather form
 // means no atomics and a result that does not depend on scheduling.
 #include "eb_internal.cuh"
 
 namespace {
 
-constexpr int kWarps = 8;
+constexpr int kThreads = 256;
 constexpr int kMaxSlots = EB_MAX_K + EB_MAX_S;
 
 __device__ __forceinline__ void fma8(float* acc, const uint4& v, float w) {
@@ -22,14 +23,15 @@ __device__ __forceinline__ void fma8(float* acc, const uint4& v, float w) {
 }
 
 template <int KS>
-__global__ void __launch_bounds__(kWarps * 32)
-combine_kernel(int n_tok, int H, int K, const uint4* __restrict__ yp, const int32_t* __restrict__ pos,
+__global__ void __launch_bounds__(kThreads)
+combine_kernel(int n_tok, int H, int K, int team, const uint4* __restrict__ yp, const int32_t* __restrict__ pos,
                const float* __restrict__ topk_w, uint4* __restrict__ out) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int t = blockIdx.x * kWarps + warp;
+  const int t = blockIdx.x * (kThreads / team) + threadIdx.x / team;   // team >= 32: a warp serves one token
   if (t >= n_tok) return;
-  int my_pos = lane < KS ? pos[(size_t)t * KS + lane] : -1;
-  float my_w = lane < K ? topk_w[(size_t)t * K + lane] : 1.0f;
+  const int lane = threadIdx.x & 31;
+  // lane s fetches slot s once per warp; the values are broadcast with shuffles
+  const int my_pos = lane < KS ? pos[(size_t)t * KS + lane] : -1;
+  const float my_w = lane < K ? topk_w[(size_t)t * K + lane] : 1.0f;
   if (__shfl_sync(0xffffffffu, my_pos, 0) < 0) return;  // micro-batch did not run: row untouched
   const int vec = H / 8;
   int p[KS];
@@ -39,7 +41,7 @@ combine_kernel(int n_tok, int H, int K, const uint4* __restrict__ yp, const int3
     p[s] = __shfl_sync(0xffffffffu, my_pos, s);
     w[s] = __shfl_sync(0xffffffffu, my_w, s);
   }
-  for (int v = lane; v < vec; v += 32) {
+  for (int v = threadIdx.x % team; v < vec; v += team) {
     uint4 r[KS];
 #pragma unroll
     for (int s = 0; s < KS; ++s) r[s] = __ldg(yp + (size_t)p[s] * vec + v);
@@ -54,7 +56,7 @@ combine_kernel(int n_tok, int H, int K, const uint4* __restrict__ yp, const int3
   }
 }
 
-typedef void (*combine_fn)(int, int, int, const uint4*, const int32_t*, const float*, uint4*);
+typedef void (*combine_fn)(int, int, int, int, const uint4*, const int32_t*, const float*, uint4*);
 
 template <int KS>
 struct Table {
@@ -88,8 +90,10 @@ extern "C" eb_status eb_combine(eb_ctx* c, void* stream, const eb_batch* batch, 
   cudaStream_t st = (cudaStream_t)stream;
   const int KS = c->cfg.K + c->cfg.S;
   KernelTimer timer(c, EBK_COMBINE, st);
-  table[KS]<<<(bp.n_tok + kWarps - 1) / kWarps, kWarps * 32, 0, st>>>(bp.n_tok, c->cfg.H, c->cfg.K, (const uint4*)yp,
-                                                                     pos, topk_w, (uint4*)out);
+  const int vec = c->cfg.H / 8;
+  const int team = vec <= 32 ? 32 : vec <= 64 ? 64 : vec <= 128 ? 128 : 256, tpb = kThreads / team;
+  table[KS]<<<(bp.n_tok + tpb - 1) / tpb, kThreads, 0, st>>>(bp.n_tok, c->cfg.H, c->cfg.K, team, (const uint4*)yp, pos,
+                                                            topk_w, (uint4*)out);
   EB_LAUNCH_CHECK(c, "combine");
   return EB_OK;
 }

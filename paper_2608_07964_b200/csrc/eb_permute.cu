@@ -54,9 +54,16 @@ __device__ __forceinline__ StepShape step_shape(const BatchParams& bp, uint32_t 
 __device__ __forceinline__ int home_start(int d, int T, int D) { return (int)(((long long)d * T + D - 1) / D); }
 
 // group id of (device d, active-layer rank lr, local slot) ; local slot < n_d + S
-__device__ __forceinline__ int group_id(const ModelParams& mp, int nl, int d, int lr, int local) {
-  int n_d = mp.dev_off[d + 1] - mp.dev_off[d];
-  return nl * (mp.dev_off[d] + d * mp.S) + lr * (n_d + mp.S) + local;
+__device__ __forceinline__ int group_id(const int* dev_off, int S, int nl, int d, int lr, int local) {
+  int n_d = dev_off[d + 1] - dev_off[d];
+  return nl * (dev_off[d] + d * S) + lr * (n_d + S) + local;
+}
+
+// Copies the per-device expert offsets into shared memory (independent loads issued together) so the
+// group decoding below does not chase dependent global loads.  Ends with a block barrier.
+__device__ __forceinline__ void stage_dev_off(const ModelParams& mp, int* s_dev_off) {
+  if (threadIdx.x <= mp.D) s_dev_off[threadIdx.x] = mp.dev_off[threadIdx.x];
+  __syncthreads();
 }
 
 __device__ __forceinline__ int mb_of_chunk(const BatchParams& bp, int c) {
@@ -95,17 +102,19 @@ __global__ void __launch_bounds__(kWarps * 32)
 sizes_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ res,
              const int32_t* __restrict__ chunk_hist, int32_t* __restrict__ chunk_base,
              int32_t* __restrict__ group_size) {
+  __shared__ int s_dev_off[EB_MAX_D + 1];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = blockIdx.x * kWarps + warp;
   const uint32_t run = res->run_mask;
+  stage_dev_off(mp, s_dev_off);
   const StepShape ss = step_shape(bp, run);
   const int G = ss.nl * (mp.E + mp.D * mp.S);
   if (g >= G) return;
   // decode g -> (d, lr, local)
   int d = 0;
-  while (d + 1 < mp.D && g >= ss.nl * (mp.dev_off[d + 1] + (d + 1) * mp.S)) ++d;
-  const int n_d = mp.dev_off[d + 1] - mp.dev_off[d];
-  const int rel = g - ss.nl * (mp.dev_off[d] + d * mp.S);
+  while (d + 1 < mp.D && g >= ss.nl * (s_dev_off[d + 1] + (d + 1) * mp.S)) ++d;
+  const int n_d = s_dev_off[d + 1] - s_dev_off[d];
+  const int rel = g - ss.nl * (s_dev_off[d] + d * mp.S);
   const int lr = rel / (n_d + mp.S), local = rel % (n_d + mp.S);
   if (local >= n_d) {
     // shared expert: rows = chosen tokens at this layer whose home device is d (closed form)
@@ -120,7 +129,7 @@ sizes_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__
     }
     return;
   }
-  const int e = mp.dev_list[mp.dev_off[d] + local];
+  const int e = mp.dev_list[s_dev_off[d] + local];
   int carry = 0;
   for (int j = 0; j < bp.n_mb; ++j) {
     if (ss.rank_of_mb[j] != lr) continue;
@@ -147,12 +156,13 @@ scan_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ 
             int32_t* __restrict__ group_w, int32_t* __restrict__ step_meta) {
   __shared__ int s_warp[32];
   __shared__ int s_carry;
+  __shared__ int s_dev_off[EB_MAX_D + 1];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t run = res->run_mask;
+  if (tid == 0) s_carry = 0;
+  stage_dev_off(mp, s_dev_off);
   const StepShape ss = step_shape(bp, run);
   const int G = ss.nl * (mp.E + mp.D * mp.S);
-  if (tid == 0) s_carry = 0;
-  __syncthreads();
   for (int base = 0; base < G; base += 1024) {
     int g = base + tid;
     int v = g < G ? group_size[g] : 0;
@@ -179,11 +189,11 @@ scan_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ 
       group_off[g] = excl;
       // weight matrix of the group
       int d = 0;
-      while (d + 1 < mp.D && g >= ss.nl * (mp.dev_off[d + 1] + (d + 1) * mp.S)) ++d;
-      int n_d = mp.dev_off[d + 1] - mp.dev_off[d];
-      int rel = g - ss.nl * (mp.dev_off[d] + d * mp.S);
+      while (d + 1 < mp.D && g >= ss.nl * (s_dev_off[d + 1] + (d + 1) * mp.S)) ++d;
+      int n_d = s_dev_off[d + 1] - s_dev_off[d];
+      int rel = g - ss.nl * (s_dev_off[d] + d * mp.S);
       int lr = rel / (n_d + mp.S), local = rel % (n_d + mp.S);
-      int slot = local < n_d ? mp.dev_list[mp.dev_off[d] + local] : mp.E + (local - n_d);
+      int slot = local < n_d ? mp.dev_list[s_dev_off[d] + local] : mp.E + (local - n_d);
       group_w[g] = ss.act_layer[lr] * (mp.E + mp.S) + slot;
     }
     __syncthreads();
@@ -196,7 +206,7 @@ scan_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ 
     step_meta[1] = G;
     step_meta[2] = ss.nl;
     for (int d = 0; d <= mp.D; ++d)
-      step_meta[3 + d] = d < mp.D ? ss.nl * (mp.dev_off[d] + d * mp.S) : G;
+      step_meta[3 + d] = d < mp.D ? ss.nl * (s_dev_off[d] + d * mp.S) : G;
     for (int i = 4 + mp.D; i < EB_META_LEN; ++i) step_meta[i] = 0;
   }
 }
@@ -207,8 +217,10 @@ rank_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ 
             const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ chunk_base,
             const int32_t* __restrict__ group_off, int32_t* __restrict__ pos, int32_t* __restrict__ row_src) {
   __shared__ int s_next[kWarps][EB_MAX_E];
+  __shared__ int s_dev_off[EB_MAX_D + 1];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int c = blockIdx.x * kWarps + warp;
+  stage_dev_off(mp, s_dev_off);
   if (c >= bp.n_chunks) return;
   const int E = mp.E, K = mp.K, S = mp.S, KS = K + S;
   const int j = mb_of_chunk(bp, c);
@@ -224,7 +236,7 @@ rank_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ 
   int* next = s_next[warp];
   for (int e = lane; e < E; e += 32) {
     int d = mp.e2d[e];
-    next[e] = group_off[group_id(mp, ss.nl, d, lr, mp.e_local[e])] + chunk_base[(size_t)c * E + e];
+    next[e] = group_off[group_id(s_dev_off, mp.S, ss.nl, d, lr, mp.e_local[e])] + chunk_base[(size_t)c * E + e];
   }
   __syncwarp();
   // routed slots, in assignment order a = t_local * K + k
@@ -256,9 +268,9 @@ rank_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ 
         int T2 = bp.tok_off[j2 + 1] - bp.tok_off[j2];
         before += home_start(d + 1, T2, mp.D) - home_start(d, T2, mp.D);
       }
-    const int n_d = mp.dev_off[d + 1] - mp.dev_off[d];
+    const int n_d = s_dev_off[d + 1] - s_dev_off[d];
     for (int s = 0; s < S; ++s) {
-      int p = group_off[group_id(mp, ss.nl, d, lr, n_d + s)] + before + (tl - home_start(d, T, mp.D));
+      int p = group_off[group_id(s_dev_off, mp.S, ss.nl, d, lr, n_d + s)] + before + (tl - home_start(d, T, mp.D));
       pos[(size_t)(t0 + lane) * KS + K + s] = p;
       row_src[p] = t0 + lane;
     }
@@ -266,35 +278,32 @@ rank_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ 
 }
 
 // ---- gather --------------------------------------------------------------------------------
-// One warp per token: the row is read once as 16-byte vectors and written to each of its rows.
-__global__ void __launch_bounds__(kWarps * 32)
-gather_kernel(int n_tok, int H, int KS, const uint4* __restrict__ x, const int32_t* __restrict__ pos,
+// A team of threads per token (one 16-byte vector each, so a whole row is in flight at once): the row
+// is read once and written to each of its K + S rows.  `team` is 32..256 and divides the block.
+constexpr int kGatherThreads = 256;
+
+__global__ void __launch_bounds__(kGatherThreads)
+gather_kernel(int n_tok, int H, int KS, int team, const uint4* __restrict__ x, const int32_t* __restrict__ pos,
               uint4* __restrict__ xp) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int t = blockIdx.x * kWarps + warp;
+  const int t = blockIdx.x * (kGatherThreads / team) + threadIdx.x / team;   // team >= 32: a warp serves one token
   if (t >= n_tok) return;
-  int my_pos = lane < KS ? pos[(size_t)t * KS + lane] : -1;
-  if (__shfl_sync(0xffffffffu, my_pos, 0) < 0) return;  // micro-batch does not run
-  const int vec = H / 8;                                // 16-byte vectors per row
+  const int lane = threadIdx.x & 31;
+  const int my_pos = lane < KS ? pos[(size_t)t * KS + lane] : -1;   // lane s fetches slot s once per warp
+  if (__shfl_sync(0xffffffffu, my_pos, 0) < 0) return;              // micro-batch does not run
+  const int vec = H / 8;  // 16-byte vectors per row
   const uint4* src = x + (size_t)t * vec;
-  for (int v0 = 0; v0 < vec; v0 += 32 * 4) {
-    uint4 r[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      int v = v0 + u * 32 + lane;
-      if (v < vec) r[u] = __ldg(src + v);
-    }
+  for (int v0 = 0; v0 < vec; v0 += team) {
+    const int v = v0 + threadIdx.x % team;
+    uint4 r = make_uint4(0, 0, 0, 0);
+    if (v < vec) r = __ldg(src + v);
     for (int s = 0; s < KS; ++s) {
-      int p = __shfl_sync(0xffffffffu, my_pos, s);
-      uint4* dst = xp + (size_t)p * vec;
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        int v = v0 + u * 32 + lane;
-        if (v < vec) dst[v] = r[u];
-      }
+      const int p = __shfl_sync(0xffffffffu, my_pos, s);
+      if (v < vec) xp[(size_t)p * vec + v] = r;
     }
   }
 }
+
+static inline int team_for(int vec) { return vec <= 32 ? 32 : vec <= 64 ? 64 : vec <= 128 ? 128 : 256; }
 
 }  // namespace
 
@@ -344,8 +353,9 @@ extern "C" eb_status eb_permute(eb_ctx* c, void* stream, const eb_batch* batch, 
   }
   if (bp.n_tok > 0) {
     KernelTimer timer(c, EBK_PERMUTE_GATHER, st);
-    gather_kernel<<<(bp.n_tok + kWarps - 1) / kWarps, kWarps * 32, 0, st>>>(
-        bp.n_tok, c->cfg.H, c->cfg.K + c->cfg.S, (const uint4*)x, pos, (uint4*)xp);
+    const int team = team_for(c->cfg.H / 8), tpb = kGatherThreads / team;
+    gather_kernel<<<(bp.n_tok + tpb - 1) / tpb, kGatherThreads, 0, st>>>(bp.n_tok, c->cfg.H, c->cfg.K + c->cfg.S, team,
+                                                                         (const uint4*)x, pos, (uint4*)xp);
   }
   EB_LAUNCH_CHECK(c, "permute");
   return EB_OK;
@@ -465,9 +475,11 @@ extern "C" eb_status eb_permute_noalloc(const eb_config* cfg, void* stream, cons
   scan_kernel<<<1, 1024, 0, st>>>(mp, bp, d_res, d_gsize, group_off, group_w, step_meta);
   if (bp.n_chunks > 0)
     rank_kernel<<<chunk_blocks, kWarps * 32, 0, st>>>(mp, bp, d_res, topk_idx, d_cbase, group_off, pos, row_src);
-  if (bp.n_tok > 0)
-    gather_kernel<<<(bp.n_tok + kWarps - 1) / kWarps, kWarps * 32, 0, st>>>(bp.n_tok, g.H, g.K + g.S, (const uint4*)x,
-                                                                            pos, (uint4*)xp);
+  if (bp.n_tok > 0) {
+    const int team = team_for(g.H / 8), tpb = kGatherThreads / team;
+    gather_kernel<<<(bp.n_tok + tpb - 1) / tpb, kGatherThreads, 0, st>>>(bp.n_tok, g.H, g.K + g.S, team, (const uint4*)x,
+                                                                         pos, (uint4*)xp);
+  }
   ce = cudaGetLastError();
   if (ce != cudaSuccess) return noalloc_fail(err, err_cap, EB_ERR_CUDA, cudaGetErrorString(ce));
   return EB_OK;
