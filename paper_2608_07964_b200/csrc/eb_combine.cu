@@ -26,6 +26,7 @@ template <int KS>
 __global__ void __launch_bounds__(kThreads)
 combine_kernel(int n_tok, int H, int K, int team, const uint4* __restrict__ yp, const int32_t* __restrict__ pos,
                const float* __restrict__ topk_w, uint4* __restrict__ out) {
+  EB_GRID_DEP_SYNC();
   const int t = blockIdx.x * (kThreads / team) + threadIdx.x / team;   // team >= 32: a warp serves one token
   if (t >= n_tok) return;
   const int lane = threadIdx.x & 31;
@@ -92,8 +93,8 @@ extern "C" eb_status eb_combine(eb_ctx* c, void* stream, const eb_batch* batch, 
   KernelTimer timer(c, EBK_COMBINE, st);
   const int vec = c->cfg.H / 8;
   const int team = vec <= 32 ? 32 : vec <= 64 ? 64 : vec <= 128 ? 128 : 256, tpb = kThreads / team;
-  table[KS]<<<(bp.n_tok + tpb - 1) / tpb, kThreads, 0, st>>>(bp.n_tok, c->cfg.H, c->cfg.K, team, (const uint4*)yp, pos,
-                                                            topk_w, (uint4*)out);
+  ebi_launch(table[KS], dim3((bp.n_tok + tpb - 1) / tpb), dim3(kThreads), 0, st, bp.n_tok, c->cfg.H, c->cfg.K, team,
+             (const uint4*)yp, pos, topk_w, (uint4*)out);
   EB_LAUNCH_CHECK(c, "combine");
   return EB_OK;
 }

@@ -224,6 +224,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
            const __grid_constant__ CUtensorMap tmB0, const __grid_constant__ CUtensorMap tmB1,
            const int4* __restrict__ work, const int32_t* __restrict__ work_count, bf16* __restrict__ out,
            int ld_out, int n_out, int k_total, int* status) {
+  EB_GRID_DEP_SYNC();
   constexpr int NS = PAIR ? kPairStages : kStages;
   constexpr int SB = PAIR ? kPairStageBytes : kStageBytes;
   extern __shared__ uint8_t smem_raw[];
@@ -450,6 +451,7 @@ __global__ void __launch_bounds__(1024)
 plan_kernel(const int32_t* __restrict__ group_off, const int32_t* __restrict__ step_meta, int device, int nt1, int nt2,
             int allow_pairs, int32_t* __restrict__ mtile_pref, int32_t* __restrict__ ptile_pref,
             int32_t* __restrict__ work_count) {
+  EB_GRID_DEP_SYNC();
   __shared__ long long s_warp[32];
   __shared__ long long s_carry;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -516,6 +518,7 @@ fill_kernel(const int32_t* __restrict__ group_off, const int32_t* __restrict__ g
             const int32_t* __restrict__ mtile_pref, const int32_t* __restrict__ ptile_pref,
             const int32_t* __restrict__ work_count, int nt1, int nt2, int max1, int max2, int maxp1, int maxp2,
             int4* __restrict__ work1, int4* __restrict__ work2, int4* __restrict__ work1p, int4* __restrict__ work2p) {
+  EB_GRID_DEP_SYNC();
   const int g0 = work_count[3], ng = work_count[4];
   const int cnt[4] = {work_count[0], work_count[1], work_count[5], work_count[6]};
   const int total = cnt[0] + cnt[1] + cnt[2] + cnt[3];
@@ -591,13 +594,15 @@ cudaError_t launch_ffn(eb_ctx* c, cudaStream_t st, const CUtensorMap& tA, const 
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = PAIR ? 2 : 1;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   const int32_t* wc = c->work_count;
   return cudaLaunchKernelEx(&cfg, ffn_kernel<PHASE, PAIR>, tA, tAs, tB0, tB1, work, wc, out, ld_out, n_out, k_total,
                             c->d_status);
@@ -665,14 +670,14 @@ eb_status ebi_ffn_run(eb_ctx* c, cudaStream_t st, const void* xp, const int32_t*
   if (pairs && c->hint_meta == step_meta && c->hint_max_group_rows >= 0 && c->hint_max_group_rows <= BM) pairs = false;
   {
     KernelTimer timer(c, EBK_FFN_PLAN, st);
-    plan_kernel<<<1, 1024, 0, st>>>(group_off, step_meta, device, nt1, nt2, pairs ? 1 : 0, c->mtile_pref, c->ptile_pref,
-                                    c->work_count);
+    ebi_launch(plan_kernel, dim3(1), dim3(1024), 0, st, group_off, step_meta, (int)device, nt1, nt2, pairs ? 1 : 0,
+               c->mtile_pref, c->ptile_pref, c->work_count);
   }
   {
     KernelTimer timer(c, EBK_FFN_FILL, st);
-    fill_kernel<<<c->num_sms, 256, 0, st>>>(group_off, group_w, c->mtile_pref, c->ptile_pref, c->work_count, nt1, nt2,
-                                            c->max_work1, c->max_work2, c->max_work1p, c->max_work2p, c->work1, c->work2,
-                                            c->work1p, c->work2p);
+    ebi_launch(fill_kernel, dim3(c->num_sms), dim3(256), 0, st, group_off, group_w, (const int32_t*)c->mtile_pref,
+               (const int32_t*)c->ptile_pref, (const int32_t*)c->work_count, nt1, nt2, c->max_work1, c->max_work2,
+               c->max_work1p, c->max_work2p, c->work1, c->work2, c->work1p, c->work2p);
   }
   cudaError_t e = cudaSuccess;
   if (pairs) {

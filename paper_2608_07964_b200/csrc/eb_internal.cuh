@@ -127,6 +127,28 @@ struct KernelTimer {
     if (_e != cudaSuccess) return ebi_check_cuda((ctx), _e, what);      \
   } while (0)
 
+// Every kernel of the library begins with EB_GRID_DEP_SYNC(): it waits until the kernels before it in
+// the stream have finished (and their writes are visible), then lets the kernel after it start being
+// scheduled.  With launches made through ebi_launch (programmatic stream serialisation) the launch
+// latency of each small kernel overlaps the previous kernel; with ordinary launches it is a no-op.
+#define EB_GRID_DEP_SYNC() asm volatile("griddepcontrol.wait;\n\tgriddepcontrol.launch_dependents;" ::: "memory")
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t ebi_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                     Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 static inline bool ebi_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Entry points of the per-step stages (defined in their own translation units).

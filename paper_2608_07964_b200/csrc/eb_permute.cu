@@ -76,6 +76,7 @@ __device__ __forceinline__ int mb_of_chunk(const BatchParams& bp, int c) {
 __global__ void __launch_bounds__(kWarps * 32)
 hist_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ res,
             const int32_t* __restrict__ topk_idx, int32_t* __restrict__ chunk_hist) {
+  EB_GRID_DEP_SYNC();
   __shared__ int s_hist[kWarps][EB_MAX_E];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int c = blockIdx.x * kWarps + warp;
@@ -102,6 +103,7 @@ __global__ void __launch_bounds__(kWarps * 32)
 sizes_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ res,
              const int32_t* __restrict__ chunk_hist, int32_t* __restrict__ chunk_base,
              int32_t* __restrict__ group_size) {
+  EB_GRID_DEP_SYNC();
   __shared__ int s_dev_off[EB_MAX_D + 1];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = blockIdx.x * kWarps + warp;
@@ -154,6 +156,7 @@ __global__ void __launch_bounds__(1024)
 scan_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ res,
             const int32_t* __restrict__ group_size, int32_t* __restrict__ group_off,
             int32_t* __restrict__ group_w, int32_t* __restrict__ step_meta) {
+  EB_GRID_DEP_SYNC();
   __shared__ int s_warp[32];
   __shared__ int s_carry;
   __shared__ int s_dev_off[EB_MAX_D + 1];
@@ -216,6 +219,7 @@ __global__ void __launch_bounds__(kWarps * 32)
 rank_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ res,
             const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ chunk_base,
             const int32_t* __restrict__ group_off, int32_t* __restrict__ pos, int32_t* __restrict__ row_src) {
+  EB_GRID_DEP_SYNC();
   __shared__ int s_next[kWarps][EB_MAX_E];
   __shared__ int s_dev_off[EB_MAX_D + 1];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -285,6 +289,7 @@ constexpr int kGatherThreads = 256;
 __global__ void __launch_bounds__(kGatherThreads)
 gather_kernel(int n_tok, int H, int KS, int team, const uint4* __restrict__ x, const int32_t* __restrict__ pos,
               uint4* __restrict__ xp) {
+  EB_GRID_DEP_SYNC();
   const int t = blockIdx.x * (kGatherThreads / team) + threadIdx.x / team;   // team >= 32: a warp serves one token
   if (t >= n_tok) return;
   const int lane = threadIdx.x & 31;
@@ -336,26 +341,28 @@ extern "C" eb_status eb_permute(eb_ctx* c, void* stream, const eb_batch* batch, 
   const int chunk_blocks = (bp.n_chunks + kWarps - 1) / kWarps;
   if (bp.n_chunks > 0) {
     KernelTimer timer(c, EBK_PERMUTE_HIST, st);
-    hist_kernel<<<chunk_blocks, kWarps * 32, 0, st>>>(c->mp, bp, d_res, topk_idx, c->chunk_hist);
+    ebi_launch(hist_kernel, dim3(chunk_blocks), dim3(kWarps * 32), 0, st, c->mp, bp, d_res, topk_idx, c->chunk_hist);
   }
   {
     KernelTimer timer(c, EBK_PERMUTE_SIZES, st);
-    sizes_kernel<<<(gcap + kWarps - 1) / kWarps, kWarps * 32, 0, st>>>(c->mp, bp, d_res, c->chunk_hist, c->chunk_base,
-                                                                        c->group_size);
+    ebi_launch(sizes_kernel, dim3((gcap + kWarps - 1) / kWarps), dim3(kWarps * 32), 0, st, c->mp, bp, d_res,
+               (const int32_t*)c->chunk_hist, c->chunk_base, c->group_size);
   }
   {
     KernelTimer timer(c, EBK_PERMUTE_SCAN, st);
-    scan_kernel<<<1, 1024, 0, st>>>(c->mp, bp, d_res, c->group_size, group_off, group_w, step_meta);
+    ebi_launch(scan_kernel, dim3(1), dim3(1024), 0, st, c->mp, bp, d_res, (const int32_t*)c->group_size, group_off, group_w,
+               step_meta);
   }
   if (bp.n_chunks > 0) {
     KernelTimer timer(c, EBK_PERMUTE_RANK, st);
-    rank_kernel<<<chunk_blocks, kWarps * 32, 0, st>>>(c->mp, bp, d_res, topk_idx, c->chunk_base, group_off, pos, row_src);
+    ebi_launch(rank_kernel, dim3(chunk_blocks), dim3(kWarps * 32), 0, st, c->mp, bp, d_res, topk_idx,
+               (const int32_t*)c->chunk_base, (const int32_t*)group_off, pos, row_src);
   }
   if (bp.n_tok > 0) {
     KernelTimer timer(c, EBK_PERMUTE_GATHER, st);
     const int team = team_for(c->cfg.H / 8), tpb = kGatherThreads / team;
-    gather_kernel<<<(bp.n_tok + tpb - 1) / tpb, kGatherThreads, 0, st>>>(bp.n_tok, c->cfg.H, c->cfg.K + c->cfg.S, team,
-                                                                         (const uint4*)x, pos, (uint4*)xp);
+    ebi_launch(gather_kernel, dim3((bp.n_tok + tpb - 1) / tpb), dim3(kGatherThreads), 0, st, bp.n_tok, c->cfg.H,
+               c->cfg.K + c->cfg.S, team, (const uint4*)x, (const int32_t*)pos, (uint4*)xp);
   }
   EB_LAUNCH_CHECK(c, "permute");
   return EB_OK;

@@ -16,6 +16,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 route_kernel(ModelParams mp, BatchParams bp, uint32_t route_mask, const float* __restrict__ logits,
              int32_t* __restrict__ topk_idx, float* __restrict__ topk_w, int32_t* __restrict__ mb_load,
              int32_t* __restrict__ mb_cnt) {
+  EB_GRID_DEP_SYNC();
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int t = blockIdx.x * kWarpsPerBlock + warp;
@@ -89,6 +90,7 @@ route_kernel(ModelParams mp, BatchParams bp, uint32_t route_mask, const float* _
 
 __global__ void route_clear_kernel(ModelParams mp, BatchParams bp, uint32_t route_mask, int32_t* mb_load,
                                    int32_t* mb_cnt) {
+  EB_GRID_DEP_SYNC();
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   int per = mp.E + mp.D;
   if (i >= bp.n_mb * per) return;
@@ -113,10 +115,11 @@ extern "C" eb_status eb_route(eb_ctx* c, void* stream, const eb_batch* batch, ui
   cudaStream_t st = (cudaStream_t)stream;
   KernelTimer timer(c, EBK_ROUTE, st);
   int n = bp.n_mb * (c->cfg.E + c->cfg.D);
-  route_clear_kernel<<<(n + 255) / 256, 256, 0, st>>>(c->mp, bp, route_mask, mb_load, mb_cnt);
+  ebi_launch(route_clear_kernel, dim3((n + 255) / 256), dim3(256), 0, st, c->mp, bp, route_mask, mb_load, mb_cnt);
   if (bp.n_tok > 0) {
     int blocks = (bp.n_tok + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    route_kernel<<<blocks, kWarpsPerBlock * 32, 0, st>>>(c->mp, bp, route_mask, logits, topk_idx, topk_w, mb_load, mb_cnt);
+    ebi_launch(route_kernel, dim3(blocks), dim3(kWarpsPerBlock * 32), 0, st, c->mp, bp, route_mask, logits, topk_idx, topk_w,
+               mb_load, mb_cnt);
   }
   EB_LAUNCH_CHECK(c, "route");
   return EB_OK;

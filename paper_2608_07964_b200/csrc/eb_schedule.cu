@@ -51,6 +51,7 @@ __device__ __forceinline__ Cand make_cand(const long long* w, int D, int n, unsi
 __global__ void __launch_bounds__(kThreads)
 schedule_kernel(int D, int n_mb, uint32_t pool_mask, int m, int policy, const int32_t* __restrict__ mb_load,
                 eb_sched_result* __restrict__ res) {
+  EB_GRID_DEP_SYNC();
   __shared__ int s_load[EB_MAX_MB][EB_MAX_D];
   __shared__ int s_lo[256][EB_MAX_D];
   __shared__ int s_hi[256][EB_MAX_D];
@@ -212,7 +213,8 @@ extern "C" eb_status eb_schedule(eb_ctx* c, void* stream, const eb_batch* batch,
   cudaStream_t st = (cudaStream_t)stream;
   {
     KernelTimer timer(c, EBK_SCHEDULE, st);
-    schedule_kernel<<<1, kThreads, 0, st>>>(c->cfg.D, bp.n_mb, batch->pool_mask, m, (int)policy, mb_load, d_res);
+    ebi_launch(schedule_kernel, dim3(1), dim3(kThreads), 0, st, c->cfg.D, bp.n_mb, batch->pool_mask, (int)m, (int)policy,
+               mb_load, d_res);
   }
   EB_LAUNCH_CHECK(c, "schedule");
   if (h_res) {
