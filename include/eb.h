@@ -238,6 +238,12 @@ eb_status eb_permute_noalloc(const eb_config* cfg, void* stream, const eb_batch*
 /* Reads (and clears) the context's device status word; synchronises the device. */
 eb_status eb_device_status(eb_ctx* ctx, int32_t* out_status);
 
+/* Exercises the bounded wait used by the expert kernels without any fault: one CTA waits on a
+ * barrier that nothing arrives on, for at most `limit_cycles` SM cycles (1 .. 2e9), then gives up,
+ * records EB_ERR_TIMEOUT in the context status word and returns normally.  *out_gave_up (host) is
+ * set to 1 if the wait expired.  Synchronises the stream.  The context stays usable. */
+eb_status eb_selftest_bounded_wait(eb_ctx* ctx, void* stream, int64_t limit_cycles, int32_t* out_gave_up);
+
 /* Per-kernel timing: when enabled every internal launch is bracketed by CUDA events on its
  * stream.  eb_kernel_ms synchronises and writes the duration in ms of the most recent launch of
  * each kernel (negative if it has not run since timing was enabled); `ms` is host [eb_num_kernels()]. */

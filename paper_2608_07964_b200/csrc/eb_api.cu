@@ -258,6 +258,19 @@ extern "C" eb_status eb_device_status(eb_ctx* c, int32_t* out_status) {
   return EB_OK;
 }
 
+extern "C" eb_status eb_selftest_bounded_wait(eb_ctx* c, void* stream, int64_t limit_cycles, int32_t* out_gave_up) {
+  if (!c || !out_gave_up) return EB_ERR_INVALID_ARG;
+  if (limit_cycles < 1 || limit_cycles > 2000000000LL) return ebi_fail(c, EB_ERR_INVALID_ARG, "limit_cycles out of range");
+  if (!c->ws) return ebi_fail(c, EB_ERR_WORKSPACE, "no workspace set");
+  cudaStream_t st = (cudaStream_t)stream;
+  int* d_flag = c->work_count + 7;   // scratch word of the workspace, rewritten by the next expert pass
+  eb_status s = ebi_selftest_wait(c, st, limit_cycles, d_flag);
+  if (s != EB_OK) return s;
+  EB_CUDA(c, cudaMemcpyAsync(out_gave_up, d_flag, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  EB_CUDA(c, cudaStreamSynchronize(st));
+  return EB_OK;
+}
+
 static const char* kKernelNames[EBK_COUNT] = {
     "route", "schedule", "permute_hist", "permute_sizes", "permute_scan", "permute_rank",
     "permute_gather", "ffn_plan", "ffn_fill", "ffn_gateup", "ffn_down", "ffn_gateup_pair", "ffn_down_pair", "combine"};

@@ -72,14 +72,15 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait: false if the limit expired or another thread of the CTA already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* s_abort, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* s_abort, int* status,
+                                          long long limit = kSpinLimitCycles) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t spin = 1;; ++spin) {
     if (mbar_try(bar, parity)) return true;
     if ((spin & 63u) == 0u) {
       if (*s_abort) return false;
-      if (clock64() - t0 > kSpinLimitCycles) {
+      if (clock64() - t0 > limit) {
         *s_abort = 1;
         atomicExch(status, (int)EB_ERR_TIMEOUT);
         return false;
@@ -436,6 +437,24 @@ done:
   }
 }
 
+// ---- self-test of the bounded wait ---------------------------------------------------------------
+// One CTA waits on a barrier that nothing ever arrives on, with a short cycle limit, through the same
+// wait routine the expert kernels use: the wait gives up, records EB_ERR_TIMEOUT and the kernel returns.
+__global__ void bounded_wait_probe_kernel(long long limit_cycles, int* status, int* gave_up) {
+  __shared__ uint64_t bar;
+  __shared__ int s_abort;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    bool ok = mbar_wait(smem_u32(&bar), 0, &s_abort, status, limit_cycles);
+    *gave_up = ok ? 0 : 1;
+  }
+}
+
 // ---- tile list construction ------------------------------------------------------------------
 // A group runs either on single CTAs (128-row tiles) or on CTA pairs (256-row tiles), never both, so
 // its weights are streamed by one kernel only.  Pairs are used when they do not add padded rows
@@ -609,6 +628,12 @@ cudaError_t launch_ffn(eb_ctx* c, cudaStream_t st, const CUtensorMap& tA, const 
 }
 
 }  // namespace
+
+eb_status ebi_selftest_wait(eb_ctx* c, cudaStream_t st, long long limit_cycles, int* d_gave_up) {
+  bounded_wait_probe_kernel<<<1, 32, 0, st>>>(limit_cycles, c->d_status, d_gave_up);
+  EB_LAUNCH_CHECK(c, "bounded wait probe");
+  return EB_OK;
+}
 
 eb_status ebi_ffn_bind(eb_ctx* c) {
   const eb_config& g = c->cfg;

@@ -155,3 +155,4 @@ static inline bool ebi_aligned16(const void* p) { return (reinterpret_cast<uintp
 eb_status ebi_ffn_run(eb_ctx* c, cudaStream_t st, const void* xp, const int32_t* group_off,
                       const int32_t* group_w, const int32_t* step_meta, void* yp, int32_t device);
 eb_status ebi_ffn_bind(eb_ctx* c);
+eb_status ebi_selftest_wait(eb_ctx* c, cudaStream_t st, long long limit_cycles, int* d_gave_up);

@@ -324,3 +324,33 @@ def test_group_sizes_around_the_pair_tile_boundaries():
     case.logits = logits[perm].contiguous()
     step, ref = _full_step(case, store, 1)
     assert sorted(np.diff(ref["group_off"]).tolist()) == sorted(sizes)
+
+
+# ----------------------------------------------------------------------------------- failure reporting
+def test_bounded_wait_gives_up_and_reports_without_harming_the_context():
+    B = _binding()
+    wl = synth.workload("c1")
+    case = Hn.make_case(wl)
+    store = Hn.WeightStore(wl)
+    step, ref = _full_step(case, store, wl.m)
+    want = step.out[:case.T_tot].clone()
+    assert step.selftest_bounded_wait(2_000_000) == 1          # the wait ran out (about a millisecond)
+    assert step.device_status() == 5                            # EB_ERR_TIMEOUT was recorded ...
+    assert step.device_status() == 0                            # ... and reading it clears it
+    batch = B.Batch(case.tok_off, case.layers)
+    step.eb_step(batch, wl.m)                                   # the context is still usable
+    torch.cuda.synchronize()
+    assert torch.equal(step.out[:case.T_tot], want)
+    assert step.device_status() == 0
+
+
+# ----------------------------------------------------------------------------------- extreme shapes
+def test_minimal_hidden_sizes_and_maximum_slots():
+    # H = I = 8 (one 16-byte vector per row) and K + S = 16 slots per token
+    wl = _small(L=2, E=16, K=8, S=8, D=4, N=3, T=20, H=8, I=8, mapping="mod")
+    _full_step(Hn.make_case(wl, [20, 1, 45], [0, 1, 1]), Hn.WeightStore(wl), 2)
+
+
+def test_sixteen_micro_batches_on_one_layer():
+    wl = _small(L=1, E=8, K=2, S=1, D=4, N=16, T=40, H=128, I=192, mapping="contiguous", zipf_s=0.3)
+    _full_step(Hn.make_case(wl, [40 + 3 * (j % 4) for j in range(16)], [0] * 16), Hn.WeightStore(wl), 12)
