@@ -32,7 +32,9 @@ from paper_2608_07964_b200 import synth  # noqa: E402
 
 METRIC = "cross-layer MoE step tokens/s"
 UNIT = "tokens/s"
-KERNELS_PER_STEP = 15  # route 2, schedule 1, permute 5, expert FFN 6 (plan, fill, 2 x gate/up, 2 x down), combine 1
+# Kernels per step: route 2, schedule 1, permute 5, expert pass 4 or 6 (plan, fill, gate/up and down on single
+# CTAs, plus their CTA-pair launches when a group can exceed 128 rows), combine 1.  bench counts them from the
+# library's own launch counter.
 
 # DRAM traffic of the dominant kernel (ffn gate/up) from an ncu capture: dram__bytes_read.sum +
 # dram__bytes_write.sum over the algorithmic bytes of the captured launch.  The capture ran on the
@@ -273,6 +275,15 @@ def run_ours(args, wl):
     batch = B.Batch(wl.tok_off, wl.layers)
     m = wl.m
     run = lambda: step.eb_step(batch, m)
+    if args.graph:
+        run()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        captured0 = B.launch_count()
+        with torch.cuda.graph(graph):
+            step.eb_step(batch, m)
+        captured = B.launch_count() - captured0     # kernel nodes of one step
+        run = graph.replay
 
     def barrier():
         torch.cuda.synchronize()
@@ -288,7 +299,11 @@ def run_ours(args, wl):
     sampler.start()
     time.sleep(0.25)
     t0 = time.time()
+    launches0 = B.launch_count()
     ms = timed(run, args.steps)
+    launches = B.launch_count() - launches0
+    if args.graph:
+        launches = captured * args.steps
     t1 = time.time()
     clocks = sampler.stop(t0, t1)
     barrier()
@@ -375,7 +390,7 @@ def run_ours(args, wl):
                 data="synthetic", config=workload_config(wl), clocks=clocks,
                 e2e=dict(value=tok_total / (ms_e2e_max / args.steps / 1e3), unit=UNIT, h2d_bytes_per_step=h2d,
                          d2h_bytes_per_step=d2h),
-                gpu_launches=KERNELS_PER_STEP * args.steps, roofline=roof, cpu_baseline=cpu,
+                gpu_launches=launches, roofline=roof, cpu_baseline=cpu,
                 tokens_per_step=tok_total, run_mask=sched["run_mask"], device_status=status, idle=idle, detail=extra)
     print(json.dumps(line))
     if dist is not None:
@@ -429,6 +444,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c2small", "c3", "c3init", "c3initsmall", "c4"])
+    ap.add_argument("--graph", action="store_true", help="replay the step from a captured CUDA graph")
     ap.add_argument("--no-idle", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

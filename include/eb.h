@@ -252,6 +252,10 @@ const char* eb_kernel_name(int32_t i);
 eb_status eb_set_timing(eb_ctx* ctx, int32_t enabled);
 eb_status eb_kernel_ms(eb_ctx* ctx, float* ms);
 
+/* Kernels launched by the library in this process so far (all contexts; launches through the
+ * allocation-free entry point and the self-test are not counted). */
+uint64_t eb_launch_count(void);
+
 const char* eb_status_string(eb_status s);
 /* Text of the last failure on this context (host string, valid until the next call). */
 const char* eb_last_error(const eb_ctx* ctx);

@@ -47,7 +47,7 @@ SYMBOLS = ["eb_create", "eb_destroy", "eb_bind_weights", "eb_workspace_bytes", "
            "eb_expert_ffn_grouped", "eb_expert_ffn_device", "eb_combine", "eb_step", "eb_step_host",
            "eb_permute_noalloc", "eb_selftest_bounded_wait",
            "eb_device_status", "eb_num_kernels", "eb_kernel_name", "eb_set_timing", "eb_kernel_ms",
-           "eb_status_string", "eb_last_error"]
+           "eb_launch_count", "eb_status_string", "eb_last_error"]
 
 _lib = None
 
@@ -91,6 +91,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.eb_kernel_name.restype = C.c_char_p
     lib.eb_set_timing.argtypes = [vp, i32]
     lib.eb_kernel_ms.argtypes = [vp, C.POINTER(C.c_float)]
+    lib.eb_launch_count.argtypes = []
+    lib.eb_launch_count.restype = C.c_uint64
     lib.eb_status_string.argtypes = [i32]
     lib.eb_status_string.restype = C.c_char_p
     lib.eb_last_error.argtypes = [vp]
@@ -301,6 +303,11 @@ def permute_noalloc(L, E, K, S, H, D, expert_to_device: Sequence[int], batch: Ba
                                   pos.data_ptr(), xp.data_ptr(), step_meta.data_ptr(), err, 256)
     if code != 0:
         raise EbError(code, lib.eb_status_string(code).decode() + ": " + err.value.decode())
+
+
+def launch_count() -> int:
+    """Kernels launched by the library in this process so far."""
+    return int(load_library().eb_launch_count())
 
 
 def _sched_dict(h: EbSchedResult, D: int) -> Dict:

@@ -6,6 +6,10 @@
 
 #include "eb_internal.cuh"
 
+unsigned long long g_ebi_launches = 0;
+
+extern "C" uint64_t eb_launch_count(void) { return g_ebi_launches; }
+
 int32_t ebi_rows_cap(const eb_ctx* c) { return c->cfg.max_tokens * (c->cfg.K + c->cfg.S); }
 int32_t ebi_groups_cap(const eb_ctx* c) { return EB_MAX_MB * (c->cfg.E + c->cfg.D * c->cfg.S); }
 

@@ -623,6 +623,7 @@ cudaError_t launch_ffn(eb_ctx* c, cudaStream_t st, const CUtensorMap& tA, const 
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   const int32_t* wc = c->work_count;
+  ++g_ebi_launches;
   return cudaLaunchKernelEx(&cfg, ffn_kernel<PHASE, PAIR>, tA, tAs, tB0, tB1, work, wc, out, ld_out, n_out, k_total,
                             c->d_status);
 }

@@ -133,6 +133,9 @@ struct KernelTimer {
 // latency of each small kernel overlaps the previous kernel; with ordinary launches it is a no-op.
 #define EB_GRID_DEP_SYNC() asm volatile("griddepcontrol.wait;\n\tgriddepcontrol.launch_dependents;" ::: "memory")
 
+// Number of kernels this library has launched in the process (all contexts).
+extern unsigned long long g_ebi_launches;
+
 template <typename... KArgs, typename... Args>
 static inline cudaError_t ebi_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
                                      Args... args) {
@@ -146,6 +149,7 @@ static inline cudaError_t ebi_launch(void (*kernel)(KArgs...), dim3 grid, dim3 b
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  ++g_ebi_launches;
   return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 

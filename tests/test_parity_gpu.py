@@ -354,3 +354,39 @@ def test_minimal_hidden_sizes_and_maximum_slots():
 def test_sixteen_micro_batches_on_one_layer():
     wl = _small(L=1, E=8, K=2, S=1, D=4, N=16, T=40, H=128, I=192, mapping="contiguous", zipf_s=0.3)
     _full_step(Hn.make_case(wl, [40 + 3 * (j % 4) for j in range(16)], [0] * 16), Hn.WeightStore(wl), 12)
+
+
+# ----------------------------------------------------------------------------------- CUDA graph
+def test_step_replayed_from_a_cuda_graph_matches_eager():
+    """The five calls only enqueue work on the stream, so a whole step can be captured once and replayed;
+    new inputs are written into the same device buffers between replays."""
+    B = _binding()
+    wl = synth.workload("c1")
+    store = Hn.WeightStore(wl)
+    step = B.from_workload(wl)
+    step.bind_weights(store.gate, store.up, store.down)
+    batch = B.Batch(wl.tok_off, wl.layers)
+    T = wl.T_tot
+    case_a = Hn.make_case(wl)
+    case_b = Hn.make_case(synth.workload("c1", seed=77))
+    step.logits[:T].copy_(case_a.logits)
+    step.x[:T].copy_(case_a.x)
+    step.eb_step(batch, wl.m)                     # warm-up outside capture (first-use set-up)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step.eb_step(batch, wl.m)
+    for case in (case_b, case_a, case_b):
+        step.logits[:T].copy_(case.logits)
+        step.x[:T].copy_(case.x)
+        step.out.fill_(-7.0)
+        graph.replay()
+        torch.cuda.synchronize()
+        replayed = step.out[:T].clone()
+        mask_replayed = step.sched_result()["run_mask"]
+        step.out.fill_(-7.0)
+        step.eb_step(batch, wl.m)
+        torch.cuda.synchronize()
+        assert step.sched_result()["run_mask"] == mask_replayed
+        assert torch.equal(step.out[:T], replayed)
+    assert step.device_status() == 0
