@@ -33,15 +33,59 @@ def timed_ms(fn, reps=5, warm=2):
     return a.elapsed_time(b) / reps
 
 
+def ep_size_sweep(args, dev, weights):
+    """Expert-parallel size sweep at constant per-device tokens (the paper's Table 4 set-up: batch grows
+    with the number of devices), N = 4 micro-batches and m = 3 as in the paper's default; plus how often a
+    micro-batch's workload peaks on the same device in N consecutive layers (the paper's Table 2 statistic).
+    Peak devices are read off the load vectors eb_route produced."""
+    lines = ["| s | D | tokens per micro-batch | idle EB (MaxUtil) | idle EB (CumUtil) | idle EB (DiffPeak) | idle alone | idle lock-step | same peak, 2 layers | same peak, 3 layers |",
+             "|---|---|---|---|---|---|---|---|---|---|"]
+    for s in (0.5, 1.0):
+        for D in (2, 4, 8):
+            wl = synth.workload_c5(4, 64 * D, s, D=D, m_override=3)
+            bias = synth.zipf_bias(wl)
+            step = B.from_workload(wl, device=dev)
+            step.bind_weights(*weights)
+            logits_of = lambda j, l: synth.logits_for(wl, j, l, dev, bias)
+            res = {}
+            for name, pol in (("max", B.POLICY_MAXUTIL), ("cum", B.POLICY_CUMUTIL), ("diff", B.POLICY_DIFFPEAK)):
+                res[name] = driver.idle_fractions(driver.run_load_trace(step, wl.tok_off, wl.L, wl.m, pol, logits_of), D)
+            lock = driver.idle_fractions(driver.run_load_trace(step, wl.tok_off, wl.L, wl.N, B.POLICY_ALL, logits_of), D)
+            # per (micro-batch, layer) peak device from the routed loads
+            peaks = {}
+            for l in range(wl.L):
+                for j in range(wl.N):
+                    step.logits[wl.tok_off[j]:wl.tok_off[j + 1]].copy_(logits_of(j, l))
+                step.eb_route(B.Batch(wl.tok_off, [l] * wl.N))
+                loads = step.mb_load[:wl.N].cpu().tolist()
+                for j in range(wl.N):
+                    peaks[(j, l)] = max(range(D), key=lambda d: (loads[j][d], -d))
+            same2 = sum(peaks[(j, l)] == peaks[(j, l + 1)] for j in range(wl.N) for l in range(wl.L - 1))
+            same3 = sum(peaks[(j, l)] == peaks[(j, l + 1)] == peaks[(j, l + 2)] for j in range(wl.N) for l in range(wl.L - 2))
+            lines.append(f"| {s} | {D} | {wl.T} | {res['max']['idle_cross_layer']:.3f} | {res['cum']['idle_cross_layer']:.3f} | "
+                         f"{res['diff']['idle_cross_layer']:.3f} | {res['max']['idle_each_alone']:.3f} | {lock['idle_cross_layer']:.3f} | "
+                         f"{same2}/{wl.N * (wl.L - 1)} | {same3}/{wl.N * (wl.L - 2)} |")
+            step.close()
+            print(lines[-1], flush=True)
+    return lines
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--out", default=None)
     ap.add_argument("--policy", type=int, default=B.POLICY_MAXUTIL)
     ap.add_argument("--quick", action="store_true", help="s in {0, 1.0}, N in {4, 16} only")
+    ap.add_argument("--ep", action="store_true", help="expert-parallel size sweep instead of the skew sweep")
     args = ap.parse_args(argv)
     dev = "cuda:0"
     base = synth.workload_c5(2, 16, 0.0)
     weights = tuple(synth.all_weights(base, k, dev) for k in ("gate", "up", "down"))
+    if args.ep:
+        text = "\n".join(ep_size_sweep(args, dev, weights)) + "\n"
+        if args.out:
+            with open(args.out, "w") as f:
+                f.write(text)
+        return 0
     svals = [0.0, 1.0] if args.quick else [0.0, 0.5, 1.0, 1.5]
     nvals = [4, 16] if args.quick else [2, 4, 8, 16]
     lines = ["| s | N | T | steps EB(.75) | idle EB m=.75N | idle EB m=.5N | idle alone | idle lock-step | step ms | step tokens/s | step run/N |",
