@@ -238,6 +238,16 @@ eb_status eb_permute_noalloc(const eb_config* cfg, void* stream, const eb_batch*
 /* Reads (and clears) the context's device status word; synchronises the device. */
 eb_status eb_device_status(eb_ctx* ctx, int32_t* out_status);
 
+/* Consistency check of a step's permutation tables on the device, for debugging without a memory
+ * checker: offsets ascending and ending at the row count, weight ids in range, pos and row_src
+ * mutually inverse on the chosen tokens and -1 elsewhere, every row in a group of its token's layer
+ * and expert, token order kept inside groups.  Every index is range-checked before it is used.
+ * Writes the number of violations to *out_errors (host) and synchronises the stream. */
+eb_status eb_check_permutation(eb_ctx* ctx, void* stream, const eb_batch* batch, const eb_sched_result* d_res,
+                               const int32_t* topk_idx, const int32_t* group_off, const int32_t* group_w,
+                               const int32_t* row_src, const int32_t* pos, const int32_t* step_meta,
+                               int32_t* out_errors);
+
 /* Exercises the bounded wait used by the expert kernels without any fault: one CTA waits on a
  * barrier that nothing arrives on, for at most `limit_cycles` SM cycles (1 .. 2e9), then gives up,
  * records EB_ERR_TIMEOUT in the context status word and returns normally.  *out_gave_up (host) is

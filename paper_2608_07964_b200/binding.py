@@ -45,7 +45,7 @@ class EbStepBuffers(C.Structure):
 SYMBOLS = ["eb_create", "eb_destroy", "eb_bind_weights", "eb_workspace_bytes", "eb_set_workspace",
            "eb_rows_capacity", "eb_groups_capacity", "eb_route", "eb_schedule", "eb_permute",
            "eb_expert_ffn_grouped", "eb_expert_ffn_device", "eb_combine", "eb_step", "eb_step_host",
-           "eb_permute_noalloc", "eb_selftest_bounded_wait",
+           "eb_permute_noalloc", "eb_selftest_bounded_wait", "eb_check_permutation",
            "eb_device_status", "eb_num_kernels", "eb_kernel_name", "eb_set_timing", "eb_kernel_ms",
            "eb_launch_count", "eb_status_string", "eb_last_error"]
 
@@ -84,6 +84,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.eb_step_host.argtypes = [vp, vp, C.POINTER(EbBatch), u32, i32, i32, C.POINTER(EbStepBuffers), vp, vp, vp, vp]
     lib.eb_permute_noalloc.argtypes = [C.POINTER(EbConfig), vp, C.POINTER(EbBatch), vp, vp, vp, vp, vp, vp, vp, vp, vp,
                                        C.c_char_p, C.c_size_t]
+    lib.eb_check_permutation.argtypes = [vp, vp, C.POINTER(EbBatch), vp, vp, vp, vp, vp, vp, vp, C.POINTER(i32)]
     lib.eb_selftest_bounded_wait.argtypes = [vp, vp, C.c_int64, C.POINTER(i32)]
     lib.eb_device_status.argtypes = [vp, C.POINTER(i32)]
     lib.eb_num_kernels.argtypes = []
@@ -270,6 +271,15 @@ class MoEStep:
     def device_status(self) -> int:
         v = C.c_int32(0)
         self._check(self.lib.eb_device_status(self.ctx, C.byref(v)))
+        return v.value
+
+    def check_permutation(self, batch: Batch) -> int:
+        """Number of inconsistencies the device-side checker finds in the tables of the last eb_permute."""
+        v = C.c_int32(-1)
+        self._check(self.lib.eb_check_permutation(self.ctx, _stream(), C.byref(batch.c), self.sched.data_ptr(),
+                                                  self.topk_idx.data_ptr(), self.group_off.data_ptr(),
+                                                  self.group_w.data_ptr(), self.row_src.data_ptr(), self.pos.data_ptr(),
+                                                  self.step_meta.data_ptr(), C.byref(v)))
         return v.value
 
     def selftest_bounded_wait(self, limit_cycles: int = 2_000_000) -> int:

@@ -468,7 +468,7 @@ __device__ __forceinline__ bool group_uses_pairs(int rows) {
 // exclusive scans of both; totals.
 __global__ void __launch_bounds__(1024)
 plan_kernel(const int32_t* __restrict__ group_off, const int32_t* __restrict__ step_meta, int device, int nt1, int nt2,
-            int allow_pairs, int32_t* __restrict__ mtile_pref, int32_t* __restrict__ ptile_pref,
+            int pair_mode, int32_t* __restrict__ mtile_pref, int32_t* __restrict__ ptile_pref,
             int32_t* __restrict__ work_count) {
   EB_GRID_DEP_SYNC();
   __shared__ long long s_warp[32];
@@ -485,7 +485,7 @@ plan_kernel(const int32_t* __restrict__ group_off, const int32_t* __restrict__ s
     long long v = 0;  // low 32 bits: single tiles, high 32 bits: pair tiles
     if (i < ng) {
       int rows = group_off[g0 + i + 1] - group_off[g0 + i];
-      if (allow_pairs && group_uses_pairs(rows)) v = (long long)((rows + 2 * BM - 1) / (2 * BM)) << 32;
+      if (pair_mode && group_uses_pairs(rows)) v = (long long)((rows + 2 * BM - 1) / (2 * BM)) << 32;
       else v = (rows + BM - 1) / BM;
     }
     long long incl = v;

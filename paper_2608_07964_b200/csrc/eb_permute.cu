@@ -368,6 +368,103 @@ extern "C" eb_status eb_permute(eb_ctx* c, void* stream, const eb_batch* batch, 
   return EB_OK;
 }
 
+// ---- eb_check_permutation ----------------------------------------------------------------------
+// Device-side consistency check of a step's permutation tables (stands in for a memory checker on
+// boxes where none is available): every index is range-checked before use, nothing is dereferenced
+// on a bad index, and the number of violations is returned.
+namespace {
+
+__global__ void __launch_bounds__(256)
+check_kernel(ModelParams mp, BatchParams bp, int rows_cap, int groups_cap, const eb_sched_result* __restrict__ res,
+             const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ group_off,
+             const int32_t* __restrict__ group_w, const int32_t* __restrict__ row_src, const int32_t* __restrict__ pos,
+             const int32_t* __restrict__ step_meta, int32_t* __restrict__ errors) {
+  EB_GRID_DEP_SYNC();
+  const int R = step_meta[0], G = step_meta[1];
+  const uint32_t run = res->run_mask;
+  const int KS = mp.K + mp.S;
+  int bad = 0;
+  const int tid = blockIdx.x * blockDim.x + threadIdx.x, nthr = gridDim.x * blockDim.x;
+  if (R < 0 || R > rows_cap || G < 0 || G > groups_cap) {
+    if (tid == 0) atomicAdd(errors, 1);
+    return;
+  }
+  // group offsets: start at 0, ascending, end at R; weight ids in range
+  for (int g = tid; g <= G; g += nthr) {
+    int o = group_off[g];
+    if (o < 0 || o > R) ++bad;
+    if (g == 0 && o != 0) ++bad;
+    if (g == G && o != R) ++bad;
+    if (g < G) {
+      if (group_off[g + 1] < o) ++bad;
+      int w = group_w[g];
+      if (w < 0 || w >= mp.L * (mp.E + mp.S)) ++bad;
+    }
+  }
+  // pos and row_src are mutually inverse on the chosen tokens; -1 elsewhere; rows land in a group of
+  // the token's layer and expert; rows of a group keep token order
+  for (int i = tid; i < bp.n_tok * KS; i += nthr) {
+    const int t = i / KS, slot = i % KS;
+    int j = 0;
+    while (j + 1 < bp.n_mb && t >= bp.tok_off[j + 1]) ++j;
+    const int p = pos[i];
+    if (!((run >> j) & 1u)) {
+      if (p != -1) ++bad;
+      continue;
+    }
+    if (p < 0 || p >= R) {
+      ++bad;
+      continue;
+    }
+    if (row_src[p] != t) ++bad;
+    // binary search of the group holding row p
+    int lo = 0, hi = G - 1;
+    while (lo < hi) {
+      int mid = (lo + hi + 1) >> 1;
+      if (group_off[mid] <= p) lo = mid; else hi = mid - 1;
+    }
+    const int w = group_w[lo];
+    const int layer = w / (mp.E + mp.S), e = w % (mp.E + mp.S);
+    if (layer != bp.layer[j]) ++bad;
+    if (slot < mp.K) {
+      const int want = topk_idx[(size_t)t * mp.K + slot];
+      if (want < 0 || want >= mp.E || e != want) ++bad;
+    } else if (e != mp.E + (slot - mp.K)) {
+      ++bad;
+    }
+    if (p > group_off[lo] && row_src[p - 1] >= t) ++bad;   // stable order inside the group
+  }
+  for (int r = tid; r < R; r += nthr) {
+    int t = row_src[r];
+    if (t < 0 || t >= bp.n_tok) ++bad;
+  }
+  if (bad) atomicAdd(errors, bad);
+}
+
+}  // namespace
+
+extern "C" eb_status eb_check_permutation(eb_ctx* c, void* stream, const eb_batch* batch, const eb_sched_result* d_res,
+                                          const int32_t* topk_idx, const int32_t* group_off, const int32_t* group_w,
+                                          const int32_t* row_src, const int32_t* pos, const int32_t* step_meta,
+                                          int32_t* out_errors) {
+  if (!c) return EB_ERR_INVALID_ARG;
+  BatchParams bp;
+  eb_status s = ebi_make_batch(c, batch, &bp);
+  if (s != EB_OK) return s;
+  if (!d_res || !topk_idx || !group_off || !group_w || !row_src || !pos || !step_meta || !out_errors)
+    return ebi_fail(c, EB_ERR_INVALID_ARG, "null pointer");
+  if (!c->ws) return ebi_fail(c, EB_ERR_WORKSPACE, "no workspace set");
+  cudaStream_t st = (cudaStream_t)stream;
+  int32_t* d_err = c->group_size;   // scratch word; the next eb_permute rewrites it
+  EB_CUDA(c, cudaMemsetAsync(d_err, 0, sizeof(int32_t), st));
+  ebi_launch(check_kernel, dim3(2 * c->num_sms), dim3(256), 0, st, c->mp, bp, ebi_rows_cap(c), ebi_groups_cap(c), d_res,
+             topk_idx, group_off, group_w, row_src, pos, step_meta, d_err);
+  EB_LAUNCH_CHECK(c, "check_permutation");
+  EB_CUDA(c, cudaMemcpyAsync(out_errors, d_err, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  EB_CUDA(c, cudaStreamSynchronize(st));
+  return EB_OK;
+}
+
 // ---- eb_permute_noalloc ------------------------------------------------------------------------
 // Same dispatch as eb_permute for callers that must not create device allocations: no context, no
 // workspace.  The expert tables and the permutation scratch live in one file-scope device array

@@ -38,6 +38,7 @@ def _full_step(case, store, m, policy=O.POLICY_MAXUTIL, pool_mask=None, check_ff
     step.eb_combine(batch)
     torch.cuda.synchronize()
     assert step.device_status() == 0
+    assert step.check_permutation(batch) == 0
 
     ref = Hn.oracle_front(case, pool, m, policy)
     Hn.check_front(step, case, ref, n_mb)
@@ -390,3 +391,29 @@ def test_step_replayed_from_a_cuda_graph_matches_eager():
         assert step.sched_result()["run_mask"] == mask_replayed
         assert torch.equal(step.out[:T], replayed)
     assert step.device_status() == 0
+
+
+def test_device_side_checker_flags_corrupted_tables():
+    B = _binding()
+    wl = synth.workload("c1")
+    case = Hn.make_case(wl)
+    step, ref = _full_step(case, Hn.WeightStore(wl), wl.m, check_ffn=False)
+    batch = B.Batch(case.tok_off, case.layers)
+    assert step.check_permutation(batch) == 0
+    t_run = int(np.nonzero(ref["pos"][:, 0] >= 0)[0][0])
+    saved = step.pos.clone()
+    step.pos[t_run, 0] = 10 ** 6                      # out of range: reported, never dereferenced
+    assert step.check_permutation(batch) > 0
+    step.pos.copy_(saved)
+    step.pos[t_run, 0], step.pos[t_run, 1] = int(saved[t_run, 1]), int(saved[t_run, 0])   # swapped slots
+    assert step.check_permutation(batch) > 0
+    step.pos.copy_(saved)
+    step.row_src[0] = -3
+    assert step.check_permutation(batch) > 0
+    assert step.device_status() == 0
+
+
+def test_c5_sweep_point_full_step():
+    # the most skewed point of the sweep with the largest micro-batch count
+    wl = synth.workload_c5(16, 128, 1.5)
+    _full_step(Hn.make_case(wl), Hn.WeightStore(wl), wl.m)
