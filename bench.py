@@ -121,14 +121,17 @@ def make_inputs(wl, device):
     return logits, x
 
 
-def algorithmic_bytes(wl, group_off, n_groups):
+def algorithmic_bytes(wl, group_off, group_w, n_groups):
+    """Bytes and flops one expert pass needs at least: every weight matrix that has rows is read once (the
+    replicas of a shared expert on the virtual devices are one matrix in memory), every row once in and out."""
     sizes = np.diff(group_off[:n_groups + 1])
     active = int((sizes > 0).sum())
+    distinct = int(len(set(group_w[:n_groups][sizes > 0].tolist())))
     R = int(sizes.sum())
     w = wl.H * wl.I * 2
-    return dict(active_groups=active, rows=R,
-                gateup=active * 2 * w + R * wl.H * 2 + R * wl.I * 2,
-                down=active * w + R * wl.I * 2 + R * wl.H * 2,
+    return dict(active_groups=active, distinct_matrices=distinct, rows=R,
+                gateup=distinct * 2 * w + R * wl.H * 2 + R * wl.I * 2,
+                down=distinct * w + R * wl.I * 2 + R * wl.H * 2,
                 gateup_flops=4.0 * wl.H * wl.I * R, down_flops=2.0 * wl.H * wl.I * R)
 
 
@@ -341,7 +344,7 @@ def run_ours(args, wl):
 
     meta = step.meta()
     goff = step.group_off.cpu().numpy()
-    alg = algorithmic_bytes(wl, goff, meta["groups"])
+    alg = algorithmic_bytes(wl, goff, step.group_w.cpu().numpy(), meta["groups"])
     ms_step = ms_max / args.steps
     value = tok_total / (ms_step / 1e3)
     # dominant kernel: the gate/up pass of the grouped expert FFN
@@ -366,7 +369,8 @@ def run_ours(args, wl):
         kernel_ms=kern_ms,
         ffn=dict(tflops=ffn_flops / t_ffn / 1e12, frac_tensor_peak=ffn_flops / t_ffn / 1e12 / peaks["tensor"],
                  gbs=ffn_bytes / t_ffn / 1e9, frac_hbm=ffn_bytes / t_ffn / 1e9 / peaks["hbm"],
-                 down_gbs=alg["down"] / t_dn / 1e9, active_groups=alg["active_groups"], rows=alg["rows"]),
+                 down_gbs=alg["down"] / t_dn / 1e9, active_groups=alg["active_groups"],
+                 distinct_matrices=alg["distinct_matrices"], rows=alg["rows"]),
         permute_gather_gbs=move / (kern_ms.get("permute_gather", float("nan")) / 1e3) / 1e9,
         combine_gbs=move / (kern_ms.get("combine", float("nan")) / 1e3) / 1e9,
     )

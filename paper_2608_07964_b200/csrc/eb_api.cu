@@ -80,7 +80,7 @@ static size_t carve(eb_ctx* c, char* base) {
   c->group_size = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
   c->mtile_pref = (int32_t*)take(sizeof(int32_t) * (size_t)(gcap + 1));
   c->ptile_pref = (int32_t*)take(sizeof(int32_t) * (size_t)(gcap + 1));
-  c->work_count = (int32_t*)take(sizeof(int32_t) * 8);
+  c->work_count = (int32_t*)take(sizeof(int32_t) * 16);
   c->work1 = (int4*)take(sizeof(int4) * (size_t)c->max_work1);
   c->work2 = (int4*)take(sizeof(int4) * (size_t)c->max_work2);
   c->work1p = (int4*)take(sizeof(int4) * (size_t)c->max_work1p);
@@ -267,7 +267,7 @@ extern "C" eb_status eb_selftest_bounded_wait(eb_ctx* c, void* stream, int64_t l
   if (limit_cycles < 1 || limit_cycles > 2000000000LL) return ebi_fail(c, EB_ERR_INVALID_ARG, "limit_cycles out of range");
   if (!c->ws) return ebi_fail(c, EB_ERR_WORKSPACE, "no workspace set");
   cudaStream_t st = (cudaStream_t)stream;
-  int* d_flag = c->work_count + 7;   // scratch word of the workspace, rewritten by the next expert pass
+  int* d_flag = c->work_count + 15;   // scratch word of the workspace
   eb_status s = ebi_selftest_wait(c, st, limit_cycles, d_flag);
   if (s != EB_OK) return s;
   EB_CUDA(c, cudaMemcpyAsync(out_gave_up, d_flag, sizeof(int32_t), cudaMemcpyDeviceToHost, st));

@@ -13,7 +13,8 @@
 // ring of {A 128x64, B 256x64} bf16 tiles in the 128-byte swizzled K-major layout; TMEM holds two
 // 128x256 fp32 accumulators so the epilogue of tile i overlaps the MMAs of tile i+1.
 // Tiles of one group are ordered weight-tile-major, so CTAs working side by side share the
-// weight tile in L2 and every weight byte leaves HBM once per group.
+// weight tile in L2 and every weight byte leaves HBM once per group; the replicas of a shared expert on
+// the virtual devices are listed next to each other for the same reason.
 // Groups with at most 32 rows load a 32-row A box (the tensor core still multiplies 128 rows,
 // the extra rows are never stored), which keeps shared-memory fill traffic close to the weight
 // bytes in the weight-streaming regime.
@@ -464,11 +465,33 @@ __device__ __forceinline__ bool group_uses_pairs(int rows) {
   return rows > BM && (rows >= 4 * BM || rem == 0 || rem > BM);
 }
 
-// plan: per group of the requested range, number of 128-row tiles or of 256-row pair tiles;
-// exclusive scans of both; totals.
+// Processing order of the groups.  The group table is device-major, so the D replicas of a shared
+// expert (one group per virtual device, all reading the same weight matrix) lie far apart in it.
+// Tiles are therefore listed in another order: first every routed group in table order, then the
+// shared groups sorted by (layer, shared expert, device), so the replicas of one matrix are worked on
+// side by side, share its tiles in L2 and the matrix leaves HBM once per step instead of D times.
+// With a device filter (per-device timing) the device's own range is listed in table order.
+__device__ __forceinline__ int group_at(const ModelParams& mp, int nl, int device, int g0, int i) {
+  if (device >= 0) return g0 + i;
+  const int routed = nl * mp.E;
+  if (i < routed) {
+    int d = 0;
+    while (d + 1 < mp.D && i >= nl * mp.dev_off[d + 1]) ++d;
+    const int n_d = mp.dev_off[d + 1] - mp.dev_off[d];
+    const int rel = i - nl * mp.dev_off[d];
+    return nl * (mp.dev_off[d] + d * mp.S) + (rel / n_d) * (n_d + mp.S) + rel % n_d;
+  }
+  const int q = i - routed;
+  const int lr = q / (mp.S * mp.D), s = (q / mp.D) % mp.S, d = q % mp.D;
+  const int n_d = mp.dev_off[d + 1] - mp.dev_off[d];
+  return nl * (mp.dev_off[d] + d * mp.S) + lr * (n_d + mp.S) + n_d + s;
+}
+
+// plan: per group (in processing order) of the requested range, number of 128-row tiles or of 256-row
+// pair tiles; exclusive scans of both; totals.
 __global__ void __launch_bounds__(1024)
-plan_kernel(const int32_t* __restrict__ group_off, const int32_t* __restrict__ step_meta, int device, int nt1, int nt2,
-            int pair_mode, int32_t* __restrict__ mtile_pref, int32_t* __restrict__ ptile_pref,
+plan_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t* __restrict__ step_meta, int device,
+            int nt1, int nt2, int pair_mode, int32_t* __restrict__ mtile_pref, int32_t* __restrict__ ptile_pref,
             int32_t* __restrict__ work_count) {
   EB_GRID_DEP_SYNC();
   __shared__ long long s_warp[32];
@@ -478,13 +501,15 @@ plan_kernel(const int32_t* __restrict__ group_off, const int32_t* __restrict__ s
   const int g0 = device < 0 ? 0 : step_meta[3 + device];
   const int g1 = device < 0 ? G : step_meta[3 + device + 1];
   const int ng = g1 - g0;
+  const int nl = step_meta[2];
   if (tid == 0) s_carry = 0;
   __syncthreads();
   for (int b = 0; b < ng; b += 1024) {
     int i = b + tid;
     long long v = 0;  // low 32 bits: single tiles, high 32 bits: pair tiles
     if (i < ng) {
-      int rows = group_off[g0 + i + 1] - group_off[g0 + i];
+      const int g = group_at(mp, nl, device, g0, i);
+      int rows = group_off[g + 1] - group_off[g];
       if (pair_mode && group_uses_pairs(rows)) v = (long long)((rows + 2 * BM - 1) / (2 * BM)) << 32;
       else v = (rows + BM - 1) / BM;
     }
@@ -524,6 +549,8 @@ plan_kernel(const int32_t* __restrict__ group_off, const int32_t* __restrict__ s
     work_count[2] = mt;
     work_count[3] = g0;
     work_count[4] = ng;
+    work_count[8] = nl;
+    work_count[9] = device;
     work_count[5] = pt * nt1;
     work_count[6] = pt * nt2;
     work_count[7] = pt;
@@ -533,12 +560,12 @@ plan_kernel(const int32_t* __restrict__ group_off, const int32_t* __restrict__ s
 // fill: one thread per tile of the four lists (single gate/up, single down, pair gate/up, pair down);
 // tiles of a group are ordered weight-tile major, row-tile minor.
 __global__ void __launch_bounds__(256)
-fill_kernel(const int32_t* __restrict__ group_off, const int32_t* __restrict__ group_w,
+fill_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t* __restrict__ group_w,
             const int32_t* __restrict__ mtile_pref, const int32_t* __restrict__ ptile_pref,
             const int32_t* __restrict__ work_count, int nt1, int nt2, int max1, int max2, int maxp1, int maxp2,
             int4* __restrict__ work1, int4* __restrict__ work2, int4* __restrict__ work1p, int4* __restrict__ work2p) {
   EB_GRID_DEP_SYNC();
-  const int g0 = work_count[3], ng = work_count[4];
+  const int g0 = work_count[3], ng = work_count[4], nl = work_count[8], device = work_count[9];
   const int cnt[4] = {work_count[0], work_count[1], work_count[5], work_count[6]};
   const int total = cnt[0] + cnt[1] + cnt[2] + cnt[3];
   for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
@@ -560,7 +587,7 @@ fill_kernel(const int32_t* __restrict__ group_off, const int32_t* __restrict__ g
     const int t_g = pref[gi + 1] - pref[gi];
     const int rem = local - pref[gi] * nt;
     const int n = rem / t_g, m = rem % t_g;
-    const int g = g0 + gi;
+    const int g = group_at(mp, nl, device, g0, gi);
     const int row0 = group_off[g] + m * tile_rows;
     int4 it;
     it.x = row0;
@@ -696,12 +723,12 @@ eb_status ebi_ffn_run(eb_ctx* c, cudaStream_t st, const void* xp, const int32_t*
   if (pairs && c->hint_meta == step_meta && c->hint_max_group_rows >= 0 && c->hint_max_group_rows <= BM) pairs = false;
   {
     KernelTimer timer(c, EBK_FFN_PLAN, st);
-    ebi_launch(plan_kernel, dim3(1), dim3(1024), 0, st, group_off, step_meta, (int)device, nt1, nt2, pairs ? 1 : 0,
+    ebi_launch(plan_kernel, dim3(1), dim3(1024), 0, st, c->mp, group_off, step_meta, (int)device, nt1, nt2, pairs ? 1 : 0,
                c->mtile_pref, c->ptile_pref, c->work_count);
   }
   {
     KernelTimer timer(c, EBK_FFN_FILL, st);
-    ebi_launch(fill_kernel, dim3(c->num_sms), dim3(256), 0, st, group_off, group_w, (const int32_t*)c->mtile_pref,
+    ebi_launch(fill_kernel, dim3(c->num_sms), dim3(256), 0, st, c->mp, group_off, group_w, (const int32_t*)c->mtile_pref,
                (const int32_t*)c->ptile_pref, (const int32_t*)c->work_count, nt1, nt2, c->max_work1, c->max_work2,
                c->max_work1p, c->max_work2p, c->work1, c->work2, c->work1p, c->work2p);
   }

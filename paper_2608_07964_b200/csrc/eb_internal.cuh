@@ -78,7 +78,7 @@ struct eb_ctx {
   int32_t* group_size = nullptr;   // [G_cap]
   int32_t* mtile_pref = nullptr;   // [G_cap + 1] 128-row tiles before each group
   int32_t* ptile_pref = nullptr;   // [G_cap + 1] 256-row pair tiles before each group
-  int32_t* work_count = nullptr;   // [8]: tile counts of the four lists, group range
+  int32_t* work_count = nullptr;   // [16]: tile counts of the four lists, group range, layers, device filter
   int4* work1 = nullptr;           // gate/up tile list
   int4* work2 = nullptr;           // down tile list
   int4* work1p = nullptr;          // gate/up tile list of the CTA-pair kernel
