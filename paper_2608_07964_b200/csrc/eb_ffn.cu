@@ -37,6 +37,8 @@ constexpr int BK = 64;
 constexpr int BN = 256;
 constexpr int kStages = 4;
 constexpr int kSmallRows = 32;
+constexpr int kMergeSlots = BM / kSmallRows;   // 32-row slots of a merged tile
+constexpr int kMergeMaxRows = 64;              // replicas of a shared expert are merged when none has more rows
 constexpr int kABytes = BM * BK * 2;
 constexpr int kASmallBytes = kSmallRows * BK * 2;
 constexpr int kBBytes = BN * BK * 2;
@@ -224,8 +226,8 @@ template <int PHASE, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA_small,
            const __grid_constant__ CUtensorMap tmB0, const __grid_constant__ CUtensorMap tmB1,
-           const int4* __restrict__ work, const int32_t* __restrict__ work_count, bf16* __restrict__ out,
-           int ld_out, int n_out, int k_total, int* status) {
+           const int4* __restrict__ work, const int2* __restrict__ slots, const int32_t* __restrict__ work_count,
+           bf16* __restrict__ out, int ld_out, int n_out, int k_total, int* status) {
   EB_GRID_DEP_SYNC();
   constexpr int NS = PAIR ? kPairStages : kStages;
   constexpr int SB = PAIR ? kPairStageBytes : kStageBytes;
@@ -286,9 +288,17 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
       int stage = 0;
       uint32_t phase = 0;
       for (int w = w_first; w < n_work; w += w_step) {
-        const int4 it = __ldg(work + w);  // x = first row, y = valid rows, z = weight matrix, w = n tile
-        const bool small = !PAIR && it.y <= kSmallRows;
-        const uint32_t tx = PAIR ? 2u * kPairStageBytes : (uint32_t)((small ? kASmallBytes : kABytes) + kBBytes);
+        // x = first row, y = valid rows, z = weight matrix, w = n tile; y < 0 marks a merged tile:
+        // -y slots of 32 rows each, described by slots[x .. x - y)
+        const int4 it = __ldg(work + w);
+        const bool merged = !PAIR && it.y < 0;
+        const int n_slots = merged ? -it.y : 0;
+        int slot_row[kMergeSlots];
+#pragma unroll
+        for (int i = 0; i < kMergeSlots; ++i) slot_row[i] = (merged && i < n_slots) ? __ldg(slots + it.x + i).x : 0;
+        const bool small = !PAIR && !merged && it.y <= kSmallRows;
+        const uint32_t tx = PAIR ? 2u * kPairStageBytes
+                                 : (uint32_t)((merged ? n_slots * kASmallBytes : small ? kASmallBytes : kABytes) + kBBytes);
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, s_abort, status)) goto done;
           const uint32_t sa = base + stage * SB, sb = sa + kABytes;
@@ -301,7 +311,13 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
             else tma_pair_load_3d(sb, &tmB0, kb * BK, it.w * BN + (int)rank * 128, it.z, fb);
           } else {
             mbar_expect_tx(full_bar(stage), tx);
-            tma_load_2d(sa, small ? &tmA_small : &tmA, kb * BK, it.x, full_bar(stage));
+            if (merged) {
+#pragma unroll
+              for (int i = 0; i < kMergeSlots; ++i)
+                if (i < n_slots) tma_load_2d(sa + i * kASmallBytes, &tmA_small, kb * BK, slot_row[i], full_bar(stage));
+            } else {
+              tma_load_2d(sa, small ? &tmA_small : &tmA, kb * BK, it.x, full_bar(stage));
+            }
             if (PHASE == 1) {
               tma_load_3d(sb, &tmB0, kb * BK, it.w * 128, it.z, full_bar(stage));
               tma_load_3d(sb + kBBytes / 2, &tmB1, kb * BK, it.w * 128, it.z, full_bar(stage));
@@ -359,11 +375,21 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
       const uint32_t aphase = (local >> 1) & 1u;
       if (!mbar_wait(tfull_bar(as), aphase, s_abort, status)) goto done;
       tc_fence_after();
-      const int r = (int)rank * BM + q * 32 + lane;   // row inside the (pair's) tile
-      const bool row_ok = r < it.y;
+      int r = (int)rank * BM + q * 32 + lane;   // row inside the (pair's) tile
+      bool row_ok = r < it.y;
+      int row_g = it.x + r;                     // row in the permuted order
+      if (!PAIR && it.y < 0) {
+        // merged tile: epilogue warp q owns slot q (32 rows of one replica group)
+        row_ok = false;
+        if (q < -it.y) {
+          const int2 sl = __ldg(slots + it.x + q);
+          row_g = sl.x + lane;
+          row_ok = lane < sl.y;
+        }
+      }
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + as * BN;
       if (PHASE == 1) {
-        bf16* dst = out + (size_t)(it.x + r) * ld_out + it.w * 128;
+        bf16* dst = out + (size_t)row_g * ld_out + it.w * 128;
         const int n_left = n_out - it.w * 128;
 #pragma unroll 1
         for (int c0 = 0; c0 < 128; c0 += 16) {
@@ -384,7 +410,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
           if (row_ok && c0 + 8 < n_left) *reinterpret_cast<uint4*>(dst + c0 + 8) = o1;
         }
       } else {
-        bf16* dst = out + (size_t)(it.x + r) * ld_out + it.w * BN;
+        bf16* dst = out + (size_t)row_g * ld_out + it.w * BN;
         const int n_left = n_out - it.w * BN;
 #pragma unroll 1
         for (int c0 = 0; c0 < BN; c0 += 32) {
@@ -487,6 +513,27 @@ __device__ __forceinline__ int group_at(const ModelParams& mp, int nl, int devic
   return nl * (mp.dev_off[d] + d * mp.S) + lr * (n_d + mp.S) + n_d + s;
 }
 
+// The D replicas of a shared expert, when all are small, are packed into common 128-row tiles: the rows
+// of each replica are cut into chunks of 32 (one TMA box, one epilogue warp), four chunks per tile, so
+// the weight tile is fetched once for all of them.  `i` is a position of the processing order; returns
+// true if it belongs to such a merged class and gives the class's first position and chunk count.
+__device__ __forceinline__ bool merged_class(const ModelParams& mp, int nl, int device, int i,
+                                             const int32_t* __restrict__ group_off, int* head, int* chunks) {
+  if (device >= 0 || mp.S == 0 || mp.D < 2 || i < nl * mp.E) return false;
+  const int q = i - nl * mp.E;
+  const int h = i - q % mp.D;   // position of the class's replica on device 0
+  int tot = 0, mx = 0;
+  for (int d = 0; d < mp.D; ++d) {
+    const int g = group_at(mp, nl, device, 0, h + d);
+    const int rows = group_off[g + 1] - group_off[g];
+    tot += (rows + kSmallRows - 1) / kSmallRows;
+    mx = rows > mx ? rows : mx;
+  }
+  *head = h;
+  *chunks = tot;
+  return mx <= kMergeMaxRows;
+}
+
 // plan: per group (in processing order) of the requested range, number of 128-row tiles or of 256-row
 // pair tiles; exclusive scans of both; totals.
 __global__ void __launch_bounds__(1024)
@@ -510,7 +557,10 @@ plan_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t
     if (i < ng) {
       const int g = group_at(mp, nl, device, g0, i);
       int rows = group_off[g + 1] - group_off[g];
-      if (pair_mode && group_uses_pairs(rows)) v = (long long)((rows + 2 * BM - 1) / (2 * BM)) << 32;
+      int head, chunks;
+      if (merged_class(mp, nl, device, i, group_off, &head, &chunks))
+        v = i == head ? (chunks + kMergeSlots - 1) / kMergeSlots : 0;   // the class's tiles sit at its first position
+      else if (pair_mode && group_uses_pairs(rows)) v = (long long)((rows + 2 * BM - 1) / (2 * BM)) << 32;
       else v = (rows + BM - 1) / BM;
     }
     long long incl = v;
@@ -563,7 +613,8 @@ __global__ void __launch_bounds__(256)
 fill_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t* __restrict__ group_w,
             const int32_t* __restrict__ mtile_pref, const int32_t* __restrict__ ptile_pref,
             const int32_t* __restrict__ work_count, int nt1, int nt2, int max1, int max2, int maxp1, int maxp2,
-            int4* __restrict__ work1, int4* __restrict__ work2, int4* __restrict__ work1p, int4* __restrict__ work2p) {
+            int4* __restrict__ work1, int4* __restrict__ work2, int4* __restrict__ work1p, int4* __restrict__ work2p,
+            int2* __restrict__ slots) {
   EB_GRID_DEP_SYNC();
   const int g0 = work_count[3], ng = work_count[4], nl = work_count[8], device = work_count[9];
   const int cnt[4] = {work_count[0], work_count[1], work_count[5], work_count[6]};
@@ -588,10 +639,30 @@ fill_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t
     const int rem = local - pref[gi] * nt;
     const int n = rem / t_g, m = rem % t_g;
     const int g = group_at(mp, nl, device, g0, gi);
-    const int row0 = group_off[g] + m * tile_rows;
     int4 it;
-    it.x = row0;
-    it.y = min(tile_rows, group_off[g + 1] - row0);
+    int head, chunks;
+    if (!pair && merged_class(mp, nl, device, gi, group_off, &head, &chunks)) {
+      // tile m of a merged class holds chunks 4m .. 4m+3 of the class (replicas in device order)
+      const int base = kMergeSlots * (pref[gi] + m);
+      const int first = kMergeSlots * m, n_here = min(kMergeSlots, chunks - first);
+      if (list == 0 && n == 0) {
+        int c = 0;   // chunks before the current replica
+        for (int d = 0; d < mp.D; ++d) {
+          const int gd = group_at(mp, nl, device, 0, head + d);
+          const int r0 = group_off[gd], rows = group_off[gd + 1] - r0;
+          const int nc = (rows + kSmallRows - 1) / kSmallRows;
+          for (int k = 0; k < nc; ++k, ++c)
+            if (c >= first && c < first + n_here)
+              slots[base + c - first] = make_int2(r0 + k * kSmallRows, min(kSmallRows, rows - k * kSmallRows));
+        }
+      }
+      it.x = base;
+      it.y = -n_here;
+    } else {
+      const int row0 = group_off[g] + m * tile_rows;
+      it.x = row0;
+      it.y = min(tile_rows, group_off[g + 1] - row0);
+    }
     it.z = group_w[g];
     it.w = n;
     int4* dst = list == 0 ? work1 : list == 1 ? work2 : list == 2 ? work1p : work2p;
@@ -635,6 +706,7 @@ bool make_map(CUtensorMap* m, const void* ptr, uint64_t d0, uint64_t d1, uint64_
 template <int PHASE, bool PAIR>
 cudaError_t launch_ffn(eb_ctx* c, cudaStream_t st, const CUtensorMap& tA, const CUtensorMap& tAs, const CUtensorMap& tB0,
                        const CUtensorMap& tB1, const int4* work, bf16* out, int ld_out, int n_out, int k_total) {
+  const int2* slots = c->slots;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(PAIR ? c->pair_grid : c->num_sms);
   cfg.blockDim = dim3(kThreads);
@@ -651,7 +723,7 @@ cudaError_t launch_ffn(eb_ctx* c, cudaStream_t st, const CUtensorMap& tA, const 
   cfg.numAttrs = 2;
   const int32_t* wc = c->work_count;
   ++g_ebi_launches;
-  return cudaLaunchKernelEx(&cfg, ffn_kernel<PHASE, PAIR>, tA, tAs, tB0, tB1, work, wc, out, ld_out, n_out, k_total,
+  return cudaLaunchKernelEx(&cfg, ffn_kernel<PHASE, PAIR>, tA, tAs, tB0, tB1, work, slots, wc, out, ld_out, n_out, k_total,
                             c->d_status);
 }
 
@@ -730,7 +802,7 @@ eb_status ebi_ffn_run(eb_ctx* c, cudaStream_t st, const void* xp, const int32_t*
     KernelTimer timer(c, EBK_FFN_FILL, st);
     ebi_launch(fill_kernel, dim3(c->num_sms), dim3(256), 0, st, c->mp, group_off, group_w, (const int32_t*)c->mtile_pref,
                (const int32_t*)c->ptile_pref, (const int32_t*)c->work_count, nt1, nt2, c->max_work1, c->max_work2,
-               c->max_work1p, c->max_work2p, c->work1, c->work2, c->work1p, c->work2p);
+               c->max_work1p, c->max_work2p, c->work1, c->work2, c->work1p, c->work2p, c->slots);
   }
   cudaError_t e = cudaSuccess;
   if (pairs) {
