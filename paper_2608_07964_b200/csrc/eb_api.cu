@@ -278,7 +278,7 @@ extern "C" eb_status eb_selftest_bounded_wait(eb_ctx* c, void* stream, int64_t l
 
 static const char* kKernelNames[EBK_COUNT] = {
     "route", "schedule", "permute_hist", "permute_sizes", "permute_scan", "permute_rank",
-    "permute_gather", "ffn_plan", "ffn_fill", "ffn_gateup", "ffn_down", "ffn_gateup_pair", "ffn_down_pair", "combine"};
+    "permute_gather", "ffn_plan", "ffn_fill", "ffn_gateup", "ffn_down", "ffn_gateup_pair", "ffn_down_pair", "combine", "permute_fused"};
 
 extern "C" int32_t eb_num_kernels(void) { return EBK_COUNT; }
 extern "C" const char* eb_kernel_name(int32_t i) { return (i >= 0 && i < EBK_COUNT) ? kKernelNames[i] : ""; }

@@ -29,6 +29,7 @@ enum EbKernel {
   EBK_FFN_GATEUP_PAIR,
   EBK_FFN_DOWN_PAIR,
   EBK_COMBINE,
+  EBK_PERMUTE_FUSED,
   EBK_COUNT
 };
 

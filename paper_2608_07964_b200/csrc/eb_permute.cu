@@ -281,6 +281,178 @@ rank_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ 
   }
 }
 
+// ---- fused kernel for small steps --------------------------------------------------------------
+// hist + sizes + scan + rank in one block when the step has at most kFusedMaxChunks chunks and
+// kFusedMaxGroups group slots: the per-chunk tables live in shared memory and three kernel boundaries
+// disappear (these kernels are pure latency on small steps).  Same arithmetic, same results.
+constexpr int kFusedMaxChunks = 32;
+constexpr int kFusedMaxGroups = 4096;
+constexpr int kFusedThreads = 1024;
+
+__global__ void __launch_bounds__(kFusedThreads)
+permute_fused_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ res,
+                     const int32_t* __restrict__ topk_idx, int32_t* __restrict__ group_off,
+                     int32_t* __restrict__ group_w, int32_t* __restrict__ pos, int32_t* __restrict__ row_src,
+                     int32_t* __restrict__ step_meta) {
+  EB_GRID_DEP_SYNC();
+  extern __shared__ int s_dyn[];
+  __shared__ int s_dev_off[EB_MAX_D + 1];
+  __shared__ int s_warp[32];
+  __shared__ int s_carry;
+  const int E = mp.E, K = mp.K, S = mp.S, KS = K + S, D = mp.D;
+  int* s_tab = s_dyn;                          // [n_chunks][E]: histogram, then first rank of the chunk in its group
+  int* s_goff = s_dyn + bp.n_chunks * E;       // [G + 1]: group sizes, then offsets
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t run = res->run_mask;
+  if (tid == 0) s_carry = 0;
+  stage_dev_off(mp, s_dev_off);
+  const StepShape ss = step_shape(bp, run);
+  const int G = ss.nl * (E + D * S);
+
+  // ---- histogram per chunk (one warp each)
+  for (int c = warp; c < bp.n_chunks; c += kFusedThreads / 32) {
+    int* h = s_tab + c * E;
+    for (int e = lane; e < E; e += 32) h[e] = 0;
+    __syncwarp();
+    const int j = mb_of_chunk(bp, c);
+    if ((run >> j) & 1u) {
+      const int t0 = bp.tok_off[j] + (c - bp.chunk_off[j]) * 32;
+      const int nt = min(32, bp.tok_off[j + 1] - t0);
+      for (int a = lane; a < nt * K; a += 32) atomicAdd(&h[topk_idx[(size_t)t0 * K + a]], 1);
+    }
+  }
+  __syncthreads();
+
+  // ---- group sizes; the chunk table turns into "rows of the group before this chunk"
+  for (int g = tid; g < G; g += kFusedThreads) {
+    int d = 0;
+    while (d + 1 < D && g >= ss.nl * (s_dev_off[d + 1] + (d + 1) * S)) ++d;
+    const int n_d = s_dev_off[d + 1] - s_dev_off[d];
+    const int rel = g - ss.nl * (s_dev_off[d] + d * S);
+    const int lr = rel / (n_d + S), local = rel % (n_d + S);
+    int tot = 0;
+    if (local >= n_d) {
+      for (int j = 0; j < bp.n_mb; ++j)
+        if (ss.rank_of_mb[j] == lr) {
+          const int T = bp.tok_off[j + 1] - bp.tok_off[j];
+          tot += home_start(d + 1, T, D) - home_start(d, T, D);
+        }
+    } else {
+      const int e = mp.dev_list[s_dev_off[d] + local];
+      for (int j = 0; j < bp.n_mb; ++j) {
+        if (ss.rank_of_mb[j] != lr) continue;
+        for (int c = bp.chunk_off[j]; c < bp.chunk_off[j + 1]; ++c) {
+          const int v = s_tab[c * E + e];
+          s_tab[c * E + e] = tot;
+          tot += v;
+        }
+      }
+    }
+    s_goff[g] = tot;
+  }
+  __syncthreads();
+
+  // ---- exclusive scan over groups, weight matrix of every group, step_meta
+  for (int base = 0; base < G; base += kFusedThreads) {
+    const int g = base + tid;
+    const int v = g < G ? s_goff[g] : 0;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int n = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += n;
+    }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      int w = s_warp[lane], wi = w;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        int n = __shfl_up_sync(0xffffffffu, wi, o);
+        if (lane >= o) wi += n;
+      }
+      s_warp[lane] = wi - w;
+    }
+    __syncthreads();
+    const int excl = s_carry + s_warp[warp] + incl - v;
+    if (g < G) {
+      s_goff[g] = excl;
+      group_off[g] = excl;
+      int d = 0;
+      while (d + 1 < D && g >= ss.nl * (s_dev_off[d + 1] + (d + 1) * S)) ++d;
+      const int n_d = s_dev_off[d + 1] - s_dev_off[d];
+      const int rel = g - ss.nl * (s_dev_off[d] + d * S);
+      const int lr = rel / (n_d + S), local = rel % (n_d + S);
+      const int slot = local < n_d ? mp.dev_list[s_dev_off[d] + local] : E + (local - n_d);
+      group_w[g] = ss.act_layer[lr] * (E + S) + slot;
+    }
+    __syncthreads();
+    if (tid == kFusedThreads - 1) s_carry = excl + v;
+    __syncthreads();
+  }
+  if (tid == 0) {
+    s_goff[G] = s_carry;
+    group_off[G] = s_carry;
+    step_meta[0] = s_carry;
+    step_meta[1] = G;
+    step_meta[2] = ss.nl;
+  }
+  if (tid >= 32 && tid < 32 + EB_META_LEN - 3) {
+    const int i = tid - 32;   // entries 3 .. EB_META_LEN-1
+    step_meta[3 + i] = i < D ? ss.nl * (s_dev_off[i] + i * S) : i == D ? G : 0;
+  }
+  __syncthreads();
+
+  // ---- ranks per chunk (one warp each), as in rank_kernel
+  for (int c = warp; c < bp.n_chunks; c += kFusedThreads / 32) {
+    const int j = mb_of_chunk(bp, c);
+    const int t0 = bp.tok_off[j] + (c - bp.chunk_off[j]) * 32;
+    const int nt = min(32, bp.tok_off[j + 1] - t0);
+    if (!((run >> j) & 1u)) {
+      for (int a = lane; a < nt * KS; a += 32) pos[(size_t)t0 * KS + a] = -1;
+      continue;
+    }
+    const int lr = ss.rank_of_mb[j];
+    int* next = s_tab + c * E;
+    for (int e = lane; e < E; e += 32)
+      next[e] += s_goff[group_id(s_dev_off, S, ss.nl, mp.e2d[e], lr, mp.e_local[e])];
+    __syncwarp();
+    for (int a0 = 0; a0 < nt * K; a0 += 32) {
+      const int a = a0 + lane;
+      const bool valid = a < nt * K;
+      const int e = valid ? topk_idx[(size_t)t0 * K + a] : -1 - lane;
+      const unsigned peers = __match_any_sync(0xffffffffu, e);
+      const int before = __popc(peers & ((1u << lane) - 1u));
+      if (valid) {
+        const int p = next[e] + before;
+        const int t = t0 + a / K, k = a % K;
+        pos[(size_t)t * KS + k] = p;
+        row_src[p] = t;
+      }
+      __syncwarp();
+      if (valid && before == 0) next[e] += __popc(peers);
+      __syncwarp();
+    }
+    if (S > 0 && lane < nt) {
+      const int T = bp.tok_off[j + 1] - bp.tok_off[j];
+      const int tl = t0 + lane - bp.tok_off[j];
+      const int d = (int)(((long long)tl * D) / T);
+      int before = 0;
+      for (int j2 = 0; j2 < j; ++j2)
+        if (ss.rank_of_mb[j2] == lr) {
+          const int T2 = bp.tok_off[j2 + 1] - bp.tok_off[j2];
+          before += home_start(d + 1, T2, D) - home_start(d, T2, D);
+        }
+      const int n_d = s_dev_off[d + 1] - s_dev_off[d];
+      for (int s2 = 0; s2 < S; ++s2) {
+        const int p = s_goff[group_id(s_dev_off, S, ss.nl, d, lr, n_d + s2)] + before + (tl - home_start(d, T, D));
+        pos[(size_t)(t0 + lane) * KS + K + s2] = p;
+        row_src[p] = t0 + lane;
+      }
+    }
+  }
+}
+
 // ---- gather --------------------------------------------------------------------------------
 // A team of threads per token (one 16-byte vector each, so a whole row is in flight at once): the row
 // is read once and written to each of its K + S rows.  `team` is 32..256 and divides the block.
@@ -339,24 +511,37 @@ extern "C" eb_status eb_permute(eb_ctx* c, void* stream, const eb_batch* batch, 
   }
   const int gcap = ebi_groups_cap(c);
   const int chunk_blocks = (bp.n_chunks + kWarps - 1) / kWarps;
-  if (bp.n_chunks > 0) {
-    KernelTimer timer(c, EBK_PERMUTE_HIST, st);
-    ebi_launch(hist_kernel, dim3(chunk_blocks), dim3(kWarps * 32), 0, st, c->mp, bp, d_res, topk_idx, c->chunk_hist);
-  }
-  {
-    KernelTimer timer(c, EBK_PERMUTE_SIZES, st);
-    ebi_launch(sizes_kernel, dim3((gcap + kWarps - 1) / kWarps), dim3(kWarps * 32), 0, st, c->mp, bp, d_res,
-               (const int32_t*)c->chunk_hist, c->chunk_base, c->group_size);
-  }
-  {
-    KernelTimer timer(c, EBK_PERMUTE_SCAN, st);
-    ebi_launch(scan_kernel, dim3(1), dim3(1024), 0, st, c->mp, bp, d_res, (const int32_t*)c->group_size, group_off, group_w,
-               step_meta);
-  }
-  if (bp.n_chunks > 0) {
-    KernelTimer timer(c, EBK_PERMUTE_RANK, st);
-    ebi_launch(rank_kernel, dim3(chunk_blocks), dim3(kWarps * 32), 0, st, c->mp, bp, d_res, topk_idx,
-               (const int32_t*)c->chunk_base, (const int32_t*)group_off, pos, row_src);
+  if (bp.n_chunks <= kFusedMaxChunks && gcap <= kFusedMaxGroups) {
+    // small step: one block does histogram, sizes, scan and ranks
+    static bool attr_set = false;
+    const size_t smem = sizeof(int) * ((size_t)kFusedMaxChunks * EB_MAX_E + kFusedMaxGroups + 1);
+    if (!attr_set) {
+      EB_CUDA(c, cudaFuncSetAttribute(permute_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      attr_set = true;
+    }
+    KernelTimer timer(c, EBK_PERMUTE_FUSED, st);
+    ebi_launch(permute_fused_kernel, dim3(1), dim3(kFusedThreads), sizeof(int) * ((size_t)bp.n_chunks * c->cfg.E + gcap + 1),
+               st, c->mp, bp, d_res, topk_idx, group_off, group_w, pos, row_src, step_meta);
+  } else {
+    if (bp.n_chunks > 0) {
+      KernelTimer timer(c, EBK_PERMUTE_HIST, st);
+      ebi_launch(hist_kernel, dim3(chunk_blocks), dim3(kWarps * 32), 0, st, c->mp, bp, d_res, topk_idx, c->chunk_hist);
+    }
+    {
+      KernelTimer timer(c, EBK_PERMUTE_SIZES, st);
+      ebi_launch(sizes_kernel, dim3((gcap + kWarps - 1) / kWarps), dim3(kWarps * 32), 0, st, c->mp, bp, d_res,
+                 (const int32_t*)c->chunk_hist, c->chunk_base, c->group_size);
+    }
+    {
+      KernelTimer timer(c, EBK_PERMUTE_SCAN, st);
+      ebi_launch(scan_kernel, dim3(1), dim3(1024), 0, st, c->mp, bp, d_res, (const int32_t*)c->group_size, group_off, group_w,
+                 step_meta);
+    }
+    if (bp.n_chunks > 0) {
+      KernelTimer timer(c, EBK_PERMUTE_RANK, st);
+      ebi_launch(rank_kernel, dim3(chunk_blocks), dim3(kWarps * 32), 0, st, c->mp, bp, d_res, topk_idx,
+                 (const int32_t*)c->chunk_base, (const int32_t*)group_off, pos, row_src);
+    }
   }
   if (bp.n_tok > 0) {
     KernelTimer timer(c, EBK_PERMUTE_GATHER, st);
