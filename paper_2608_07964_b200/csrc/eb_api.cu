@@ -135,7 +135,9 @@ extern "C" eb_status eb_create(const eb_config* cfg, eb_ctx** out) {
   bool ok = cudaMalloc(&c->d_tables, tab.size() * sizeof(int32_t)) == cudaSuccess &&
             cudaMemcpy(c->d_tables, tab.data(), tab.size() * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess &&
             cudaMalloc(&c->d_status, sizeof(int32_t)) == cudaSuccess &&
-            cudaMemset(c->d_status, 0, sizeof(int32_t)) == cudaSuccess;
+            cudaMemset(c->d_status, 0, sizeof(int32_t)) == cudaSuccess &&
+            cudaMalloc(&c->d_sched_scratch, 4096) == cudaSuccess &&
+            cudaMemset(c->d_sched_scratch, 0, 4096) == cudaSuccess;
   for (int i = 0; ok && i < 2 * EBK_COUNT; ++i) ok = cudaEventCreate(&c->ev[i]) == cudaSuccess;
   if (!ok) {
     eb_destroy(c);
@@ -157,6 +159,7 @@ extern "C" eb_status eb_destroy(eb_ctx* c) {
   if (!c) return EB_ERR_INVALID_ARG;
   if (c->d_tables) cudaFree(c->d_tables);
   if (c->d_status) cudaFree(c->d_status);
+  if (c->d_sched_scratch) cudaFree(c->d_sched_scratch);
   for (int i = 0; i < 2 * EBK_COUNT; ++i)
     if (c->ev[i]) cudaEventDestroy(c->ev[i]);
   delete c;

@@ -60,6 +60,7 @@ struct eb_ctx {
   int32_t* d_tables = nullptr;  // e2d | dev_off | dev_list | e_local
   ModelParams mp;
   int32_t* d_status = nullptr;
+  char* d_sched_scratch = nullptr;  // per-block candidates and arrival counter of the multi-block scheduler
 
   const bf16* w_gate = nullptr;
   const bf16* w_up = nullptr;

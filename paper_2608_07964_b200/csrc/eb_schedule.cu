@@ -7,11 +7,14 @@
 // candidates are compared exactly by cross-multiplying sum and max in 64-bit integers.
 // Total order: higher utilisation, then more members, then the numerically smaller mask.
 // CumUtil / DiffPeak (Section 5.2) are sequential and run on one thread.
+#include <algorithm>
+
 #include "eb_internal.cuh"
 
 namespace {
 
 constexpr int kThreads = 1024;
+constexpr int kMaxBlocks = 64;
 
 struct Cand {
   long long num;   // sum_d W_d  (D if there is no work: U := 1)
@@ -50,8 +53,9 @@ __device__ __forceinline__ Cand make_cand(const long long* w, int D, int n, unsi
 
 __global__ void __launch_bounds__(kThreads)
 schedule_kernel(int D, int n_mb, uint32_t pool_mask, int m, int policy, const int32_t* __restrict__ mb_load,
-                eb_sched_result* __restrict__ res) {
+                eb_sched_result* __restrict__ res, Cand* __restrict__ block_best, unsigned* __restrict__ block_counter) {
   EB_GRID_DEP_SYNC();
+  __shared__ bool s_last;
   __shared__ int s_load[EB_MAX_MB][EB_MAX_D];
   __shared__ int s_lo[256][EB_MAX_D];
   __shared__ int s_hi[256][EB_MAX_D];
@@ -92,7 +96,7 @@ schedule_kernel(int D, int n_mb, uint32_t pool_mask, int m, int policy, const in
     Cand best;
     best.n = -1; best.num = 0; best.peak = 1; best.sub = 0;
     const unsigned total = 1u << np, lomask = (1u << nlo) - 1u;
-    for (unsigned sub = tid + 1; sub < total; sub += kThreads) {
+    for (unsigned sub = blockIdx.x * kThreads + tid + 1; sub < total; sub += gridDim.x * kThreads) {
       int n = __popc(sub);
       if (n < m) continue;
       long long w[EB_MAX_D];
@@ -114,9 +118,46 @@ schedule_kernel(int D, int n_mb, uint32_t pool_mask, int m, int policy, const in
     }
     if ((tid & 31) == 0) s_best[tid >> 5] = best;
     __syncthreads();
+    if (gridDim.x > 1) {
+      // every block leaves its best candidate in global memory; the block that arrives last reduces them
+      // (the total order makes the result independent of which block that is)
+      if (tid == 0) {
+        Cand b = s_best[0];
+        for (int i = 1; i < kThreads / 32; ++i)
+          if (better(s_best[i], b)) b = s_best[i];
+        block_best[blockIdx.x] = b;
+        __threadfence();
+        const unsigned arrived = atomicAdd(block_counter, 1u);
+        s_last = arrived == gridDim.x - 1;
+      }
+      __syncthreads();
+      if (!s_last) return;
+      __threadfence();
+      if (tid < 32) {
+        Cand b;
+        b.n = -1; b.num = 0; b.peak = 1; b.sub = 0;
+        for (int i = tid; i < (int)gridDim.x; i += 32) {
+          const Cand o = block_best[i];
+          if (better(o, b)) b = o;
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+          Cand oth;
+          oth.num = __shfl_xor_sync(0xffffffffu, b.num, o);
+          oth.peak = __shfl_xor_sync(0xffffffffu, b.peak, o);
+          oth.n = __shfl_xor_sync(0xffffffffu, b.n, o);
+          oth.sub = __shfl_xor_sync(0xffffffffu, b.sub, o);
+          if (better(oth, b)) b = oth;
+        }
+        if (tid == 0) {
+          s_best[0] = b;
+          *block_counter = 0;   // ready for the next call
+        }
+      }
+      __syncthreads();
+    }
     if (tid == 0) {
       Cand b = s_best[0];
-      for (int i = 1; i < kThreads / 32; ++i)
+      for (int i = 1; gridDim.x == 1 && i < kThreads / 32; ++i)
         if (better(s_best[i], b)) b = s_best[i];
       uint32_t mask = 0;
       for (int k = 0; k < np; ++k)
@@ -212,9 +253,15 @@ extern "C" eb_status eb_schedule(eb_ctx* c, void* stream, const eb_batch* batch,
   if ((int)policy < 0 || (int)policy > EB_POLICY_ALL) return ebi_fail(c, EB_ERR_INVALID_ARG, "unknown policy");
   cudaStream_t st = (cudaStream_t)stream;
   {
+    // MaxUtil over a large pool: the subsets are split over several blocks (one SM cannot enumerate 2^16
+    // subsets quickly); everything else is one block
+    int np = 0;
+    for (int j = 0; j < bp.n_mb; ++j) np += (batch->pool_mask >> j) & 1u;
+    int blocks = 1;
+    if (policy == EB_POLICY_MAXUTIL && np > m && np > 11) blocks = std::min(kMaxBlocks, 1 << (np - 10));
     KernelTimer timer(c, EBK_SCHEDULE, st);
-    ebi_launch(schedule_kernel, dim3(1), dim3(kThreads), 0, st, c->cfg.D, bp.n_mb, batch->pool_mask, (int)m, (int)policy,
-               mb_load, d_res);
+    ebi_launch(schedule_kernel, dim3(blocks), dim3(kThreads), 0, st, c->cfg.D, bp.n_mb, batch->pool_mask, (int)m,
+               (int)policy, mb_load, d_res, (Cand*)c->d_sched_scratch, (unsigned*)(c->d_sched_scratch + kMaxBlocks * sizeof(Cand)));
   }
   EB_LAUNCH_CHECK(c, "schedule");
   if (h_res) {
