@@ -80,6 +80,8 @@ static size_t carve(eb_ctx* c, char* base) {
   c->group_size = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
   c->mtile_pref = (int32_t*)take(sizeof(int32_t) * (size_t)(gcap + 1));
   c->ptile_pref = (int32_t*)take(sizeof(int32_t) * (size_t)(gcap + 1));
+  c->pgroup = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
+  c->pchunks = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
   c->work_count = (int32_t*)take(sizeof(int32_t) * 16);
   c->work1 = (int4*)take(sizeof(int4) * (size_t)c->max_work1);
   c->work2 = (int4*)take(sizeof(int4) * (size_t)c->max_work2);

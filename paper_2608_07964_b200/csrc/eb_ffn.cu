@@ -497,34 +497,34 @@ __device__ __forceinline__ bool group_uses_pairs(int rows) {
 // shared groups sorted by (layer, shared expert, device), so the replicas of one matrix are worked on
 // side by side, share its tiles in L2 and the matrix leaves HBM once per step instead of D times.
 // With a device filter (per-device timing) the device's own range is listed in table order.
-__device__ __forceinline__ int group_at(const ModelParams& mp, int nl, int device, int g0, int i) {
+__device__ __forceinline__ int group_at(const ModelParams& mp, const int* dev_off, int nl, int device, int g0, int i) {
   if (device >= 0) return g0 + i;
   const int routed = nl * mp.E;
   if (i < routed) {
     int d = 0;
-    while (d + 1 < mp.D && i >= nl * mp.dev_off[d + 1]) ++d;
-    const int n_d = mp.dev_off[d + 1] - mp.dev_off[d];
-    const int rel = i - nl * mp.dev_off[d];
-    return nl * (mp.dev_off[d] + d * mp.S) + (rel / n_d) * (n_d + mp.S) + rel % n_d;
+    while (d + 1 < mp.D && i >= nl * dev_off[d + 1]) ++d;
+    const int n_d = dev_off[d + 1] - dev_off[d];
+    const int rel = i - nl * dev_off[d];
+    return nl * (dev_off[d] + d * mp.S) + (rel / n_d) * (n_d + mp.S) + rel % n_d;
   }
   const int q = i - routed;
   const int lr = q / (mp.S * mp.D), s = (q / mp.D) % mp.S, d = q % mp.D;
-  const int n_d = mp.dev_off[d + 1] - mp.dev_off[d];
-  return nl * (mp.dev_off[d] + d * mp.S) + lr * (n_d + mp.S) + n_d + s;
+  const int n_d = dev_off[d + 1] - dev_off[d];
+  return nl * (dev_off[d] + d * mp.S) + lr * (n_d + mp.S) + n_d + s;
 }
 
 // The D replicas of a shared expert, when all are small, are packed into common 128-row tiles: the rows
 // of each replica are cut into chunks of 32 (one TMA box, one epilogue warp), four chunks per tile, so
 // the weight tile is fetched once for all of them.  `i` is a position of the processing order; returns
 // true if it belongs to such a merged class and gives the class's first position and chunk count.
-__device__ __forceinline__ bool merged_class(const ModelParams& mp, int nl, int device, int i,
+__device__ __forceinline__ bool merged_class(const ModelParams& mp, const int* dev_off, int nl, int device, int i,
                                              const int32_t* __restrict__ group_off, int* head, int* chunks) {
   if (device >= 0 || mp.S == 0 || mp.D < 2 || i < nl * mp.E) return false;
   const int q = i - nl * mp.E;
   const int h = i - q % mp.D;   // position of the class's replica on device 0
   int tot = 0, mx = 0;
   for (int d = 0; d < mp.D; ++d) {
-    const int g = group_at(mp, nl, device, 0, h + d);
+    const int g = group_at(mp, dev_off, nl, device, 0, h + d);
     const int rows = group_off[g + 1] - group_off[g];
     tot += (rows + kSmallRows - 1) / kSmallRows;
     mx = rows > mx ? rows : mx;
@@ -539,11 +539,13 @@ __device__ __forceinline__ bool merged_class(const ModelParams& mp, int nl, int 
 __global__ void __launch_bounds__(1024)
 plan_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t* __restrict__ step_meta, int device,
             int nt1, int nt2, int pair_mode, int32_t* __restrict__ mtile_pref, int32_t* __restrict__ ptile_pref,
-            int32_t* __restrict__ work_count) {
+            int32_t* __restrict__ pgroup, int32_t* __restrict__ pchunks, int32_t* __restrict__ work_count) {
   EB_GRID_DEP_SYNC();
   __shared__ long long s_warp[32];
   __shared__ long long s_carry;
+  __shared__ int s_dev_off[EB_MAX_D + 1];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid <= mp.D) s_dev_off[tid] = mp.dev_off[tid];
   const int G = step_meta[1];
   const int g0 = device < 0 ? 0 : step_meta[3 + device];
   const int g1 = device < 0 ? G : step_meta[3 + device + 1];
@@ -555,13 +557,19 @@ plan_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t
     int i = b + tid;
     long long v = 0;  // low 32 bits: single tiles, high 32 bits: pair tiles
     if (i < ng) {
-      const int g = group_at(mp, nl, device, g0, i);
+      const int g = group_at(mp, s_dev_off, nl, device, g0, i);
       int rows = group_off[g + 1] - group_off[g];
       int head, chunks;
-      if (merged_class(mp, nl, device, i, group_off, &head, &chunks))
+      pgroup[i] = g;
+      pchunks[i] = -1;
+      if (merged_class(mp, s_dev_off, nl, device, i, group_off, &head, &chunks)) {
         v = i == head ? (chunks + kMergeSlots - 1) / kMergeSlots : 0;   // the class's tiles sit at its first position
-      else if (pair_mode && group_uses_pairs(rows)) v = (long long)((rows + 2 * BM - 1) / (2 * BM)) << 32;
-      else v = (rows + BM - 1) / BM;
+        pchunks[i] = chunks;
+      } else if (pair_mode && group_uses_pairs(rows)) {
+        v = (long long)((rows + 2 * BM - 1) / (2 * BM)) << 32;
+      } else {
+        v = (rows + BM - 1) / BM;
+      }
     }
     long long incl = v;
 #pragma unroll
@@ -612,11 +620,12 @@ plan_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t
 __global__ void __launch_bounds__(256)
 fill_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t* __restrict__ group_w,
             const int32_t* __restrict__ mtile_pref, const int32_t* __restrict__ ptile_pref,
+            const int32_t* __restrict__ pgroup, const int32_t* __restrict__ pchunks,
             const int32_t* __restrict__ work_count, int nt1, int nt2, int max1, int max2, int maxp1, int maxp2,
             int4* __restrict__ work1, int4* __restrict__ work2, int4* __restrict__ work1p, int4* __restrict__ work2p,
             int2* __restrict__ slots) {
   EB_GRID_DEP_SYNC();
-  const int g0 = work_count[3], ng = work_count[4], nl = work_count[8], device = work_count[9];
+  const int ng = work_count[4];
   const int cnt[4] = {work_count[0], work_count[1], work_count[5], work_count[6]};
   const int total = cnt[0] + cnt[1] + cnt[2] + cnt[3];
   for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
@@ -638,17 +647,17 @@ fill_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t
     const int t_g = pref[gi + 1] - pref[gi];
     const int rem = local - pref[gi] * nt;
     const int n = rem / t_g, m = rem % t_g;
-    const int g = group_at(mp, nl, device, g0, gi);
+    const int g = pgroup[gi];
     int4 it;
-    int head, chunks;
-    if (!pair && merged_class(mp, nl, device, gi, group_off, &head, &chunks)) {
+    const int head = gi, chunks = pchunks[gi];   // only the first position of a merged class owns tiles
+    if (!pair && chunks >= 0) {
       // tile m of a merged class holds chunks 4m .. 4m+3 of the class (replicas in device order)
       const int base = kMergeSlots * (pref[gi] + m);
       const int first = kMergeSlots * m, n_here = min(kMergeSlots, chunks - first);
       if (list == 0 && n == 0) {
         int c = 0;   // chunks before the current replica
         for (int d = 0; d < mp.D; ++d) {
-          const int gd = group_at(mp, nl, device, 0, head + d);
+          const int gd = pgroup[head + d];
           const int r0 = group_off[gd], rows = group_off[gd + 1] - r0;
           const int nc = (rows + kSmallRows - 1) / kSmallRows;
           for (int k = 0; k < nc; ++k, ++c)
@@ -796,12 +805,13 @@ eb_status ebi_ffn_run(eb_ctx* c, cudaStream_t st, const void* xp, const int32_t*
   {
     KernelTimer timer(c, EBK_FFN_PLAN, st);
     ebi_launch(plan_kernel, dim3(1), dim3(1024), 0, st, c->mp, group_off, step_meta, (int)device, nt1, nt2, pairs ? 1 : 0,
-               c->mtile_pref, c->ptile_pref, c->work_count);
+               c->mtile_pref, c->ptile_pref, c->pgroup, c->pchunks, c->work_count);
   }
   {
     KernelTimer timer(c, EBK_FFN_FILL, st);
     ebi_launch(fill_kernel, dim3(c->num_sms), dim3(256), 0, st, c->mp, group_off, group_w, (const int32_t*)c->mtile_pref,
-               (const int32_t*)c->ptile_pref, (const int32_t*)c->work_count, nt1, nt2, c->max_work1, c->max_work2,
+               (const int32_t*)c->ptile_pref, (const int32_t*)c->pgroup, (const int32_t*)c->pchunks,
+               (const int32_t*)c->work_count, nt1, nt2, c->max_work1, c->max_work2,
                c->max_work1p, c->max_work2p, c->work1, c->work2, c->work1p, c->work2p, c->slots);
   }
   cudaError_t e = cudaSuccess;
