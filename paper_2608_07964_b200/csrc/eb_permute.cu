@@ -51,7 +51,41 @@ __device__ __forceinline__ StepShape step_shape(const BatchParams& bp, uint32_t 
 }
 
 // first token (local index) of micro-batch of T tokens whose home device is >= d
-__device__ __forceinline__ int home_start(int d, int T, int D) { return (int)(((long long)d * T + D - 1) / D); }
+__device__ __forceinline__ int home_start(int d, int T, int D) {
+  if (T < (1 << 26)) return (int)(((unsigned)d * (unsigned)T + (unsigned)(D - 1)) / (unsigned)D);   // d <= 16: no overflow
+  return (int)(((long long)d * T + D - 1) / D);
+}
+// home device of local token tl of a micro-batch of T tokens: floor(tl * D / T)
+__device__ __forceinline__ int home_device(int tl, int T, int D) {
+  if (T < (1 << 26)) return (int)(((unsigned)tl * (unsigned)D) / (unsigned)T);
+  return (int)(((long long)tl * D) / T);
+}
+
+// Block-cooperative version of step_shape: threads 0..15 each place one micro-batch, the result lands in
+// shared memory.  Ends with a block barrier.
+__device__ __forceinline__ void step_shape_block(const BatchParams& bp, uint32_t run, StepShape* out) {
+  const int j = threadIdx.x;
+  if (j < EB_MAX_MB) {
+    const bool sel = j < bp.n_mb && ((run >> j) & 1u);
+    int below = 0, total = 0;
+    bool first_of_layer = sel;
+    for (int i = 0; i < bp.n_mb; ++i) {
+      if (!((run >> i) & 1u)) continue;
+      bool first = true;   // is i the first chosen micro-batch sitting at its layer?
+      for (int i2 = 0; i2 < i; ++i2)
+        if (((run >> i2) & 1u) && bp.layer[i2] == bp.layer[i]) first = false;
+      if (first) {
+        ++total;
+        if (sel && bp.layer[i] < bp.layer[j]) ++below;
+      }
+      if (sel && i < j && bp.layer[i] == bp.layer[j]) first_of_layer = false;
+    }
+    out->rank_of_mb[j] = sel ? below : -1;
+    if (first_of_layer) out->act_layer[below] = bp.layer[j];
+    if (j == 0) out->nl = total;
+  }
+  __syncthreads();
+}
 
 // group id of (device d, active-layer rank lr, local slot) ; local slot < n_d + S
 __device__ __forceinline__ int group_id(const int* dev_off, int S, int nl, int d, int lr, int local) {
@@ -108,8 +142,9 @@ sizes_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = blockIdx.x * kWarps + warp;
   const uint32_t run = res->run_mask;
-  stage_dev_off(mp, s_dev_off);
-  const StepShape ss = step_shape(bp, run);
+  __shared__ StepShape ss;
+  if (threadIdx.x <= mp.D) s_dev_off[threadIdx.x] = mp.dev_off[threadIdx.x];
+  step_shape_block(bp, run, &ss);
   const int G = ss.nl * (mp.E + mp.D * mp.S);
   if (g >= G) return;
   // decode g -> (d, lr, local)
@@ -162,9 +197,10 @@ scan_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ 
   __shared__ int s_dev_off[EB_MAX_D + 1];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t run = res->run_mask;
+  __shared__ StepShape ss;
   if (tid == 0) s_carry = 0;
-  stage_dev_off(mp, s_dev_off);
-  const StepShape ss = step_shape(bp, run);
+  if (tid <= mp.D) s_dev_off[tid] = mp.dev_off[tid];
+  step_shape_block(bp, run, &ss);
   const int G = ss.nl * (mp.E + mp.D * mp.S);
   for (int base = 0; base < G; base += 1024) {
     int g = base + tid;
@@ -224,18 +260,19 @@ rank_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ 
   __shared__ int s_dev_off[EB_MAX_D + 1];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int c = blockIdx.x * kWarps + warp;
-  stage_dev_off(mp, s_dev_off);
+  const uint32_t run = res->run_mask;
+  __shared__ StepShape ss;
+  if (threadIdx.x <= mp.D) s_dev_off[threadIdx.x] = mp.dev_off[threadIdx.x];
+  step_shape_block(bp, run, &ss);
   if (c >= bp.n_chunks) return;
   const int E = mp.E, K = mp.K, S = mp.S, KS = K + S;
   const int j = mb_of_chunk(bp, c);
-  const uint32_t run = res->run_mask;
   const int t0 = bp.tok_off[j] + (c - bp.chunk_off[j]) * 32;
   const int nt = min(32, bp.tok_off[j + 1] - t0);
   if (!((run >> j) & 1u)) {
     for (int a = lane; a < nt * KS; a += 32) pos[(size_t)t0 * KS + a] = -1;
     return;
   }
-  const StepShape ss = step_shape(bp, run);
   const int lr = ss.rank_of_mb[j];
   int* next = s_next[warp];
   for (int e = lane; e < E; e += 32) {
@@ -265,7 +302,7 @@ rank_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ 
   if (S > 0 && lane < nt) {
     const int T = bp.tok_off[j + 1] - bp.tok_off[j];
     const int tl = t0 + lane - bp.tok_off[j];
-    const int d = (int)(((long long)tl * mp.D) / T);
+    const int d = home_device(tl, T, mp.D);
     int before = 0;
     for (int j2 = 0; j2 < j; ++j2)
       if (ss.rank_of_mb[j2] == lr) {
@@ -304,9 +341,10 @@ permute_fused_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __re
   int* s_goff = s_dyn + bp.n_chunks * E;       // [G + 1]: group sizes, then offsets
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t run = res->run_mask;
+  __shared__ StepShape ss;
   if (tid == 0) s_carry = 0;
-  stage_dev_off(mp, s_dev_off);
-  const StepShape ss = step_shape(bp, run);
+  if (tid <= D) s_dev_off[tid] = mp.dev_off[tid];
+  step_shape_block(bp, run, &ss);
   const int G = ss.nl * (E + D * S);
 
   // ---- histogram per chunk (one warp each)
@@ -436,7 +474,7 @@ permute_fused_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __re
     if (S > 0 && lane < nt) {
       const int T = bp.tok_off[j + 1] - bp.tok_off[j];
       const int tl = t0 + lane - bp.tok_off[j];
-      const int d = (int)(((long long)tl * D) / T);
+      const int d = home_device(tl, T, D);
       int before = 0;
       for (int j2 = 0; j2 < j; ++j2)
         if (ss.rank_of_mb[j2] == lr) {
