@@ -107,3 +107,68 @@ def idle_fractions(steps: List[Dict], D: int) -> Dict[str, float]:
         alone = D * sum(max(w) for s in steps for w in s["member_loads"].values())
         out["idle_each_alone"] = (1.0 - work / alone) if alone else 0.0
     return out
+
+
+def _device_times(step: "B.MoEStep", D: int, reps: int = 3) -> List[float]:
+    """Median CUDA-event time (ms) of the expert pass restricted to each virtual device's groups."""
+    out = []
+    for d in range(D):
+        step.eb_expert_ffn_grouped(device=d)                       # warm the path
+        ts = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            step.eb_expert_ffn_grouped(device=d)
+            b.record()
+            b.synchronize()
+            ts.append(a.elapsed_time(b))
+        out.append(sorted(ts)[len(ts) // 2])
+    return out
+
+
+def run_emulated_latency(step: "B.MoEStep", tok_off: List[int], L: int, D: int, m: int, policy: int,
+                         logits_of: Callable[[int, int], torch.Tensor], x0: torch.Tensor,
+                         alone: bool = False) -> Dict:
+    """Expert-parallel latency of a whole run as the virtual devices would see it.
+
+    Every step is routed, scheduled and permuted by the library; the expert pass is then timed on each
+    virtual device's groups by itself, and a step costs the slowest device (the others idle until the
+    gather, Section 2.3).  Returns the summed step latency, the summed busy time and the resulting
+    time-based under-utilisation 1 - sum(busy) / (D * sum(max)).  With `alone` every (micro-batch,
+    layer) workload is executed by itself (no combination at all)."""
+    N = len(tok_off) - 1
+    T = tok_off[-1]
+    layer = [0] * N
+    pool = (1 << N) - 1 if L > 0 else 0
+    route_mask = pool
+    step.x[:T].copy_(x0)
+    lat = busy = 0.0
+    n_steps = 0
+    while pool:
+        for j in range(N):
+            if (route_mask >> j) & 1:
+                step.logits[tok_off[j]:tok_off[j + 1]].copy_(logits_of(j, layer[j]))
+        lay = [min(l, L - 1) for l in layer]
+        if route_mask:
+            step.eb_route(B.Batch(tok_off, lay, pool), route_mask)
+        if alone:
+            j0 = min(j for j in range(N) if (pool >> j) & 1 and layer[j] == min(layer[i] for i in range(N) if (pool >> i) & 1))
+            batch = B.Batch(tok_off, lay, 1 << j0)
+            run = step.eb_schedule(batch, 1, B.POLICY_ALL, to_host=True)["run_mask"]
+        else:
+            batch = B.Batch(tok_off, lay, pool)
+            run = step.eb_schedule(batch, m, policy, to_host=True)["run_mask"]
+        step.eb_permute(batch)
+        t = _device_times(step, D)
+        lat += max(t)
+        busy += sum(t)
+        n_steps += 1
+        route_mask = 0
+        for j in range(N):
+            if (run >> j) & 1:
+                layer[j] += 1
+                if layer[j] >= L:
+                    pool &= ~(1 << j)
+                else:
+                    route_mask |= 1 << j
+    return dict(steps=n_steps, latency_ms=lat, busy_ms=busy, idle_time=1.0 - busy / (D * lat) if lat else 0.0)

@@ -70,14 +70,53 @@ def ep_size_sweep(args, dev, weights):
     return lines
 
 
+def latency_report(args, dev):
+    """Emulated expert-parallel MoE latency of a whole Algorithm-1 run: cross-layer scheduling (the three
+    policies) against lock-step execution and against every workload alone; per step the cost is the
+    slowest virtual device's expert pass."""
+    lines = ["| shape | N x T | policy | steps | MoE latency ms (sum of slowest device) | time idle | vs alone | vs lock-step |",
+             "|---|---|---|---|---|---|---|---|"]
+    shapes = [("c5 s=1.0 (64 experts, top-6, 8 layers)", synth.workload_c5(4, 1024, 1.0, m_override=3)),
+              ("c5 s=1.0", synth.workload_c5(8, 512, 1.0)),
+              ("c4 cut to 8 layers (8 experts, top-2, H 4096, I 14336)", synth.workload("c4", L=8, N=4, T=2048, m_override=3))]
+    for label, wl in shapes:
+        bias = synth.zipf_bias(wl)
+        step = B.from_workload(wl, device=dev)
+        weights = tuple(synth.all_weights(wl, k, dev) for k in ("gate", "up", "down"))
+        step.bind_weights(*weights)
+        logits_of = lambda j, l: synth.logits_for(wl, j, l, dev, bias)
+        x0 = torch.cat([synth.hidden_for(wl, j, 0, dev) for j in range(wl.N)], 0)
+        res = {}
+        res["alone"] = driver.run_emulated_latency(step, wl.tok_off, wl.L, wl.D, 1, B.POLICY_ALL, logits_of, x0, alone=True)
+        res["lock-step"] = driver.run_emulated_latency(step, wl.tok_off, wl.L, wl.D, wl.N, B.POLICY_ALL, logits_of, x0)
+        for name, pol in (("MaxUtil", B.POLICY_MAXUTIL), ("CumUtil", B.POLICY_CUMUTIL), ("DiffPeak", B.POLICY_DIFFPEAK)):
+            res[name] = driver.run_emulated_latency(step, wl.tok_off, wl.L, wl.D, wl.m, pol, logits_of, x0)
+        for name, r in res.items():
+            lines.append(f"| {label} | {wl.N} x {wl.T} | {name} | {r['steps']} | {r['latency_ms']:.2f} | {r['idle_time']:.3f} | "
+                         f"{r['latency_ms'] / res['alone']['latency_ms']:.2f} | {r['latency_ms'] / res['lock-step']['latency_ms']:.2f} |")
+            print(lines[-1], flush=True)
+        assert step.device_status() == 0
+        step.close()
+        del weights
+        torch.cuda.empty_cache()
+    return lines
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--out", default=None)
     ap.add_argument("--policy", type=int, default=B.POLICY_MAXUTIL)
     ap.add_argument("--quick", action="store_true", help="s in {0, 1.0}, N in {4, 16} only")
     ap.add_argument("--ep", action="store_true", help="expert-parallel size sweep instead of the skew sweep")
+    ap.add_argument("--latency", action="store_true", help="emulated expert-parallel latency of whole runs")
     args = ap.parse_args(argv)
     dev = "cuda:0"
+    if args.latency:
+        text = "\n".join(latency_report(args, dev)) + "\n"
+        if args.out:
+            with open(args.out, "w") as f:
+                f.write(text)
+        return 0
     base = synth.workload_c5(2, 16, 0.0)
     weights = tuple(synth.all_weights(base, k, dev) for k in ("gate", "up", "down"))
     if args.ep:
