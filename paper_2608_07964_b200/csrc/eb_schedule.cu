@@ -6,7 +6,8 @@
 // Utilisation (Eq. 3 for one step) is sum(W) / (D * max(W)); D is common to all candidates, so
 // candidates are compared exactly by cross-multiplying sum and max in 64-bit integers.
 // Total order: higher utilisation, then more members, then the numerically smaller mask.
-// CumUtil / DiffPeak (Section 5.2) are sequential and run on one thread.
+// CumUtil / DiffPeak (Section 5.2) are sequential and run on one thread; topping their result up to m
+// members scores the remaining pool members in parallel, one lane each.
 #include <algorithm>
 
 #include "eb_internal.cuh"
@@ -62,6 +63,9 @@ schedule_kernel(int D, int n_mb, uint32_t pool_mask, int m, int policy, const in
   __shared__ int s_member[EB_MAX_MB];
   __shared__ Cand s_best[kThreads / 32];
   __shared__ uint32_t s_run;
+  __shared__ uint32_t s_seq_run;
+  __shared__ int s_seq_n;
+  __shared__ long long s_seq_w[EB_MAX_D];
 
   const int tid = threadIdx.x;
   for (int i = tid; i < EB_MAX_MB * EB_MAX_D; i += kThreads) {
@@ -196,28 +200,45 @@ schedule_kernel(int D, int n_mb, uint32_t pool_mask, int m, int policy, const in
         ++n;
       }
     }
-    // top up to m members: repeatedly add the member whose inclusion gives the highest utilisation
-    while (n < m) {
-      int bj = -1;
-      Cand bu;
-      bu.n = -1; bu.num = 0; bu.peak = 1; bu.sub = 0;
-      for (int k = 0; k < np; ++k) {
-        int j = s_member[k];
-        if ((run >> j) & 1u) continue;
-        long long w2[EB_MAX_D];
-        for (int d = 0; d < EB_MAX_D; ++d) w2[d] = w[d] + s_load[j][d];
-        Cand cu = make_cand(w2, D, 0, 0);
-        if (bj < 0 || cu.num * bu.peak > bu.num * cu.peak) {
-          bj = j;
-          bu = cu;
+    s_seq_run = run;
+    s_seq_n = n;
+    for (int d = 0; d < EB_MAX_D; ++d) s_seq_w[d] = w[d];
+  }
+  if (policy == EB_POLICY_CUMUTIL || policy == EB_POLICY_DIFFPEAK) {
+    if (!(np <= m)) {
+      // top up to m members: repeatedly add the member whose inclusion gives the highest utilisation
+      // (lowest index on ties); lane k of warp 0 scores pool member k
+      __syncthreads();
+      if (tid < 32) {
+        uint32_t run = s_seq_run;
+        int n = s_seq_n;
+        while (n < m) {
+          Cand cu;
+          cu.n = -1; cu.num = 0; cu.peak = 1; cu.sub = 0;
+          if (tid < np && !((run >> s_member[tid]) & 1u)) {
+            long long w2[EB_MAX_D];
+            for (int d = 0; d < EB_MAX_D; ++d) w2[d] = s_seq_w[d] + s_load[s_member[tid]][d];
+            cu = make_cand(w2, D, 1, (unsigned)tid);   // equal sizes: ties fall to the lower index
+          }
+          for (int o = 16; o > 0; o >>= 1) {
+            Cand oth;
+            oth.num = __shfl_xor_sync(0xffffffffu, cu.num, o);
+            oth.peak = __shfl_xor_sync(0xffffffffu, cu.peak, o);
+            oth.n = __shfl_xor_sync(0xffffffffu, cu.n, o);
+            oth.sub = __shfl_xor_sync(0xffffffffu, cu.sub, o);
+            if (better(oth, cu)) cu = oth;
+          }
+          if (cu.n < 0) break;
+          const int bj = s_member[cu.sub];
+          __syncwarp();
+          if (tid < EB_MAX_D) s_seq_w[tid] += s_load[bj][tid];
+          __syncwarp();
+          run |= 1u << bj;
+          ++n;
         }
+        if (tid == 0) s_run = run;
       }
-      if (bj < 0) break;
-      for (int d = 0; d < EB_MAX_D; ++d) w[d] += s_load[bj][d];
-      run |= 1u << bj;
-      ++n;
     }
-    s_run = run;
   }
   __syncthreads();
   if (tid == 0) {

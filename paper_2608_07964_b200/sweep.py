@@ -102,6 +102,25 @@ def latency_report(args, dev):
     return lines
 
 
+def schedule_latency_report(args, dev):
+    """Time of one Schedule(S, m) call per policy (CUDA events, mean of 200 back-to-back calls) on routed
+    loads of the 64-expert shape; the paper's Table 3 reports 0.13-0.28 ms per step on its host."""
+    lines = ["| micro-batches N | m | MaxUtil us | CumUtil us | DiffPeak us |", "|---|---|---|---|---|"]
+    for N in (4, 8, 16):
+        wl = synth.workload_c5(N, 128, 1.0)
+        step = B.from_workload(wl, device=dev)
+        step.logits[:wl.T_tot].copy_(synth.packed_logits(wl, device=dev))
+        batch = B.Batch(wl.tok_off, wl.layers)
+        step.eb_route(batch)
+        row = []
+        for pol in (B.POLICY_MAXUTIL, B.POLICY_CUMUTIL, B.POLICY_DIFFPEAK):
+            row.append(1000.0 * timed_ms(lambda: step.eb_schedule(batch, wl.m, pol), reps=200, warm=5))
+        lines.append(f"| {N} | {wl.m} | {row[0]:.1f} | {row[1]:.1f} | {row[2]:.1f} |")
+        print(lines[-1], flush=True)
+        step.close()
+    return lines
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--out", default=None)
@@ -109,8 +128,15 @@ def main(argv=None):
     ap.add_argument("--quick", action="store_true", help="s in {0, 1.0}, N in {4, 16} only")
     ap.add_argument("--ep", action="store_true", help="expert-parallel size sweep instead of the skew sweep")
     ap.add_argument("--latency", action="store_true", help="emulated expert-parallel latency of whole runs")
+    ap.add_argument("--sched", action="store_true", help="time of one scheduling call per policy")
     args = ap.parse_args(argv)
     dev = "cuda:0"
+    if args.sched:
+        text = "\n".join(schedule_latency_report(args, dev)) + "\n"
+        if args.out:
+            with open(args.out, "w") as f:
+                f.write(text)
+        return 0
     if args.latency:
         text = "\n".join(latency_report(args, dev)) + "\n"
         if args.out:
