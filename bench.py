@@ -447,7 +447,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c2small", "c3", "c3init", "c3initsmall", "c4"])
+    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c2small", "c3", "c3init", "c3initsmall", "c4", "c4small"])
     ap.add_argument("--graph", action="store_true", help="replay the step from a captured CUDA graph")
     ap.add_argument("--no-idle", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -460,6 +460,10 @@ def main():
         # c3init with the model cut to 2 layers (2.3 GB of weights): same kernels and tile shapes, small enough for ncu
         wl = synth.workload("c3", L=2, layers_override=tuple([0] * 16))
         wl = synth.Workload(**{**wl.__dict__, "name": "c3initsmall"})
+    elif args.workload == "c4small":
+        # the large-expert shape cut to 2 layers and 2 micro-batches (5.6 GB of weights): small enough for ncu
+        wl = synth.workload("c4", L=2, N=2, m_override=2)
+        wl = synth.Workload(**{**wl.__dict__, "name": "c4small"})
     elif args.workload == "c2small":
         # the decode shape cut to 6 layers and 6 micro-batches (6.6 GB of weights): the case ncu captures run on
         wl = synth.workload("c2", L=6, N=6)
