@@ -250,7 +250,9 @@ def workload_config(wl):
     return dict(workload=f"{wl.name}: L={wl.L} E={wl.E} K={wl.K} S={wl.S} H={wl.H} I={wl.I} D={wl.D} "
                          f"map={wl.mapping} N={wl.N}x{wl.T} tokens at layers {wl.layers} m={wl.m} zipf_s={wl.zipf_s}",
                 policy="MaxUtil", seed=wl.seed,
-                l2="inputs larger than L2: each step streams the touched expert weights (GBs) from HBM")
+                l2=("inputs larger than L2: each step streams the touched expert weights (GBs) from HBM"
+                    if wl.weight_bytes() > (1 << 30) else
+                    "small workload: all weights fit in L2 and no flush is done, figures are L2-warm"))
 
 
 # ----------------------------------------------------------------------------------------------
@@ -260,11 +262,16 @@ def run_ours(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     dist = None
+    local = local % max(1, torch.cuda.device_count())
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+        if args.dist_backend == "nccl":
+            dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+        else:
+            dist.init_process_group(args.dist_backend)
     torch.cuda.set_device(local)
     device = f"cuda:{local}"
+    red_device = device if args.dist_backend == "nccl" else "cpu"   # where the timing reductions live
     wl = replica_workload(wl, rank)
     peaks = measured_peaks()
 
@@ -336,7 +343,7 @@ def run_ours(args, wl):
     barrier()
 
     # ---- reductions over ranks
-    ms_max, ms_e2e_max, tok_total = reduce_over_ranks(dist, device, ms, ms_e2e, float(tokens_run))
+    ms_max, ms_e2e_max, tok_total = reduce_over_ranks(dist, red_device, ms, ms_e2e, float(tokens_run))
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -449,6 +456,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c2small", "c3", "c3init", "c3initsmall", "c4", "c4small"])
     ap.add_argument("--graph", action="store_true", help="replay the step from a captured CUDA graph")
+    ap.add_argument("--dist-backend", default="nccl", choices=["nccl", "gloo"],
+                    help="process-group backend for the barrier and the timing reductions (replicas share no data)")
     ap.add_argument("--no-idle", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
