@@ -158,22 +158,28 @@ eb_status eb_route(eb_ctx* ctx, void* stream, const eb_batch* batch, uint32_t ro
 eb_status eb_schedule(eb_ctx* ctx, void* stream, const eb_batch* batch, int32_t m, eb_policy policy,
                       const int32_t* mb_load, eb_sched_result* d_res, eb_sched_result* h_res);
 
-/* Dispatch on one GPU (Section 2.2): histogram of the chosen micro-batches' assignments per
+/* Dispatch on one GPU (Section 2.2; stands in for the first all-to-all): histogram of the chosen micro-batches' assignments per
  * group, exclusive prefix sum, stable ranks, and a 16-byte-vector gather of the token rows into
  * group-contiguous order.  Reads the run mask from d_res on the device.
  * x bf16 [T_tot, H]; group_off i32 [G+1]; group_w i32 [G] = layer * (E+S) + slot, the weight
  * matrix of each group; row_src i32 [R] = source token of each row; pos i32 [T_tot, K+S] = row
  * of each (token, slot), -1 for tokens of micro-batches that do not run; xp bf16 [R, H];
  * step_meta i32 [EB_META_LEN].  Buffers must have the capacities given by
- * eb_groups_capacity / eb_rows_capacity. */
+ * eb_groups_capacity / eb_rows_capacity; all are written by the call and owned by the caller.
+ * Needs a workspace (EB_ERR_WORKSPACE otherwise). */
 eb_status eb_permute(eb_ctx* ctx, void* stream, const eb_batch* batch, const eb_sched_result* d_res,
                      const void* x, const int32_t* topk_idx,
                      int32_t* group_off, int32_t* group_w, int32_t* row_src, int32_t* pos,
                      void* xp, int32_t* step_meta);
 
-/* expert_i of Eq. 1 for every group in one pass: yp[r] = W_down (silu(W_gate xp[r]) * (W_up xp[r]))
- * with the weight matrices of the row's group; bf16 in, fp32 accumulation on the tensor cores,
- * the intermediate rounded once to bf16.  xp must have eb_rows_capacity rows allocated. */
+/* expert_i of Eq. 1 for every group in one pass (the joint execution of Section 4.1):
+ * yp[r] = W_down (silu(W_gate xp[r]) * (W_up xp[r])) with the weight matrices of the row's group
+ * (group_w); bf16 in, fp32 accumulation on the tensor cores, the intermediate rounded once to bf16.
+ * group_off, group_w, step_meta are the tables eb_permute wrote (device, read only); xp bf16
+ * [eb_rows_capacity, H] and yp bf16 [eb_rows_capacity, H] must be allocated to that capacity (tiles
+ * are fetched in boxes of up to 128 rows; rows beyond the step's row count are read but never
+ * written).  Needs bound weights (else EB_ERR_INVALID_ARG) and a workspace (else EB_ERR_WORKSPACE);
+ * a tensor-map or launch failure gives EB_ERR_CUDA. */
 eb_status eb_expert_ffn_grouped(eb_ctx* ctx, void* stream, const void* xp, const int32_t* group_off,
                                 const int32_t* group_w, const int32_t* step_meta, void* yp);
 
