@@ -336,10 +336,13 @@ def run_ours(args, wl):
     h_x = x.cpu().pin_memory()
     h_out = torch.empty((T, wl.H), dtype=torch.bfloat16).pin_memory()
     run_host = lambda: step.eb_step_host(batch, m, h_logits, h_x, h_out)
-    for _ in range(min(args.warmup, 3)):
-        run_host()
-    barrier()
-    ms_e2e = timed(run_host, args.steps)
+    side = torch.cuda.Stream()      # a stream of its own: the legacy default stream adds implicit synchronisation
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for _ in range(max(args.warmup, 3)):
+            run_host()
+        barrier()
+        ms_e2e = timed(run_host, args.steps)
     barrier()
 
     # ---- reductions over ranks

@@ -752,9 +752,8 @@ eb_status ebi_ffn_bind(eb_ctx* c) {
       !make_map(&c->tm_down, c->w_down, g.I, g.H, nw, BK, BN) ||
       !make_map(&c->tm_down_half, c->w_down, g.I, g.H, nw, BK, 128))
     return ebi_fail(c, EB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the weights");
-  static bool attr_set = false;
-  static int pair_grid = 0;
-  if (!attr_set) {
+  int pair_grid = 0;
+  {   // per context: function attributes and cluster occupancy belong to the current device
     cudaError_t e = cudaFuncSetAttribute(ffn_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
@@ -779,7 +778,6 @@ eb_status ebi_ffn_bind(eb_ctx* c) {
       clusters = 0;   // pairs unavailable: every group runs on single CTAs
     }
     pair_grid = 2 * (clusters < c->num_sms / 2 ? clusters : c->num_sms / 2);
-    attr_set = true;
   }
   c->pair_grid = pair_grid;
   return EB_OK;

@@ -91,6 +91,7 @@ struct eb_ctx {
   bf16* act = nullptr;             // [R_cap][I]
   int32_t max_chunks = 0, max_mtiles = 0, max_work1 = 0, max_work2 = 0, max_work1p = 0, max_work2p = 0;
 
+  bool fused_attr_set = false;
   bool timing = false;
   cudaEvent_t ev[2 * EBK_COUNT] = {};
   bool ev_valid[EBK_COUNT] = {};

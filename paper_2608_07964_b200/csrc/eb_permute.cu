@@ -551,11 +551,10 @@ extern "C" eb_status eb_permute(eb_ctx* c, void* stream, const eb_batch* batch, 
   const int chunk_blocks = (bp.n_chunks + kWarps - 1) / kWarps;
   if (bp.n_chunks <= kFusedMaxChunks && gcap <= kFusedMaxGroups) {
     // small step: one block does histogram, sizes, scan and ranks
-    static bool attr_set = false;
     const size_t smem = sizeof(int) * ((size_t)kFusedMaxChunks * EB_MAX_E + kFusedMaxGroups + 1);
-    if (!attr_set) {
+    if (!c->fused_attr_set) {   // per context: function attributes belong to the current device
       EB_CUDA(c, cudaFuncSetAttribute(permute_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-      attr_set = true;
+      c->fused_attr_set = true;
     }
     KernelTimer timer(c, EBK_PERMUTE_FUSED, st);
     ebi_launch(permute_fused_kernel, dim3(1), dim3(kFusedThreads), sizeof(int) * ((size_t)bp.n_chunks * c->cfg.E + gcap + 1),

@@ -266,6 +266,26 @@ def test_step_and_step_host_match_the_five_calls():
     res = step.eb_step_host(batch, wl.m, h_logits, h_x, h_out)
     assert res["run_mask"] == ref["sched"]["run_mask"]
     assert torch.equal(h_out, want.cpu())
+    # repeated identical calls on a side stream: same results, and new contents of the same host buffers
+    # are picked up
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for rep in range(4):
+            if rep == 2:
+                h_x.copy_(torch.flip(case.x, dims=[0]))
+            h_out.fill_(-7.0)
+            res = step.eb_step_host(batch, wl.m, h_logits, h_x, h_out)
+            assert res["run_mask"] == ref["sched"]["run_mask"]
+            if rep < 2:
+                assert torch.equal(h_out, want.cpu())
+            else:
+                assert not torch.equal(h_out, want.cpu())
+        flipped = h_out.clone()
+    step.x[:T].copy_(torch.flip(case.x, dims=[0]))
+    step.out.fill_(-7.0)
+    step.eb_step(batch, wl.m)
+    torch.cuda.synchronize()
+    assert torch.equal(step.out[:T].cpu(), flipped)
 
 
 def test_deferred_micro_batch_keeps_its_routing():
