@@ -378,11 +378,14 @@ def run_ours(args, wl):
     extra = dict(
         kernel_ms=kern_ms,
         ffn=dict(tflops=ffn_flops / t_ffn / 1e12, frac_tensor_peak=ffn_flops / t_ffn / 1e12 / peaks["tensor"],
+                 frac_tensor_sustained=ffn_flops / t_ffn / 1e12 / peaks["tensor_sustained"],
                  gbs=ffn_bytes / t_ffn / 1e9, frac_hbm=ffn_bytes / t_ffn / 1e9 / peaks["hbm"],
                  down_gbs=alg["down"] / t_dn / 1e9, active_groups=alg["active_groups"],
                  distinct_matrices=alg["distinct_matrices"], rows=alg["rows"]),
         permute_gather_gbs=move / (kern_ms.get("permute_gather", float("nan")) / 1e3) / 1e9,
         combine_gbs=move / (kern_ms.get("combine", float("nan")) / 1e3) / 1e9,
+        permute_gather_frac_hbm=move / (kern_ms.get("permute_gather", float("nan")) / 1e3) / 1e9 / peaks["hbm"],
+        combine_frac_hbm=move / (kern_ms.get("combine", float("nan")) / 1e3) / 1e9 / peaks["hbm"],
     )
     idle = idle_report(step, batch, wl, sched, B) if world == 1 and not args.no_idle else None
 
