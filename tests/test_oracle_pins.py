@@ -55,6 +55,12 @@ def test_single_step_examples(ex):
         assert Fraction(n, d) == Fraction(*ex["idle_each_alone"])
 
 
+def test_home_device_examples():
+    for case in EXAMPLES["home_device"]["cases"]:
+        got = [O.home_device(t, case["T"], case["D"]) for t in range(case["T"])]
+        assert got == case["home"]
+
+
 @pytest.mark.parametrize("ex", EXAMPLES["driver"], ids=lambda e: e["name"])
 def test_driver_examples(ex):
     table = {tuple(int(v) for v in k.split(",")): v for k, v in ex["loads"].items()}
