@@ -419,7 +419,8 @@ def idle_report(step, batch, wl, sched, B):
 
     Token based: 1 - sum(W) / (D max(W)) from the routed loads.  Time based: the expert pass is run
     on each virtual device's contiguous group range by itself (median of 5) and the same formula is
-    applied to the times; 'per layer' runs every chosen micro-batch's workload alone."""
+    applied to the times (expert-pass kernels only, from the library's per-kernel events); 'per layer' runs
+    every chosen micro-batch's workload alone."""
     D = wl.D
     run = [j for j in range(wl.N) if (sched["run_mask"] >> j) & 1]
     loads = step.mb_load[:wl.N].cpu().numpy().astype(np.int64)
@@ -428,13 +429,8 @@ def idle_report(step, batch, wl, sched, B):
     alone_cap = D * sum(int(loads[j].max()) for j in run)
     tok_alone = 1.0 - joint.sum() / alone_cap if alone_cap else 0.0
 
-    def device_times():
-        out = []
-        for d in range(D):
-            f = lambda: step.eb_expert_ffn_grouped(device=d)
-            f()
-            out.append(statistics.median(timed(f, 1) for _ in range(5)))
-        return out
+    from paper_2608_07964_b200 import driver
+    device_times = lambda: driver.device_times(step, D, reps=5)
 
     step.eb_step(batch, wl.m)
     t_cross = device_times()

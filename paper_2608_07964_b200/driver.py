@@ -109,20 +109,23 @@ def idle_fractions(steps: List[Dict], D: int) -> Dict[str, float]:
     return out
 
 
-def _device_times(step: "B.MoEStep", D: int, reps: int = 3) -> List[float]:
-    """Median CUDA-event time (ms) of the expert pass restricted to each virtual device's groups."""
+def device_times(step: "B.MoEStep", D: int, reps: int = 3) -> List[float]:
+    """Median time (ms) of the expert-pass kernels (gate/up and down, single-CTA and CTA-pair launches)
+    restricted to each virtual device's groups, from the library's per-kernel CUDA events; the tile-list
+    construction that precedes them is not counted."""
     out = []
-    for d in range(D):
-        step.eb_expert_ffn_grouped(device=d)                       # warm the path
-        ts = []
-        for _ in range(reps):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            step.eb_expert_ffn_grouped(device=d)
-            b.record()
-            b.synchronize()
-            ts.append(a.elapsed_time(b))
-        out.append(sorted(ts)[len(ts) // 2])
+    step.set_timing(True)
+    try:
+        for d in range(D):
+            step.eb_expert_ffn_grouped(device=d)                   # warm the path
+            ts = []
+            for _ in range(reps):
+                step.eb_expert_ffn_grouped(device=d)
+                k = step.kernel_ms()
+                ts.append(sum(v for name, v in k.items() if name.startswith(("ffn_gateup", "ffn_down"))))
+            out.append(sorted(ts)[len(ts) // 2])
+    finally:
+        step.set_timing(False)
     return out
 
 
@@ -159,7 +162,7 @@ def run_emulated_latency(step: "B.MoEStep", tok_off: List[int], L: int, D: int, 
             batch = B.Batch(tok_off, lay, pool)
             run = step.eb_schedule(batch, m, policy, to_host=True)["run_mask"]
         step.eb_permute(batch)
-        t = _device_times(step, D)
+        t = device_times(step, D)
         lat += max(t)
         busy += sum(t)
         n_steps += 1
