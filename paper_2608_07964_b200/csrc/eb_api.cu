@@ -87,7 +87,7 @@ static size_t carve(eb_ctx* c, char* base) {
   c->work2 = (int4*)take(sizeof(int4) * (size_t)c->max_work2);
   c->work1p = (int4*)take(sizeof(int4) * (size_t)c->max_work1p);
   c->work2p = (int4*)take(sizeof(int4) * (size_t)c->max_work2p);
-  c->slots = (int2*)take(sizeof(int2) * 4 * (size_t)c->max_mtiles);
+  c->slots = (int2*)take(sizeof(int2) * 8 * (size_t)c->max_mtiles);
   c->act = (bf16*)take(sizeof(bf16) * (size_t)rows * g.I);
   return off;
 }

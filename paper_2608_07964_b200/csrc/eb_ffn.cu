@@ -15,7 +15,8 @@
 // Tiles of one group are ordered weight-tile-major, so CTAs working side by side share the
 // weight tile in L2 and every weight byte leaves HBM once per group; the replicas of a shared expert on
 // the virtual devices are listed next to each other for the same reason.
-// Groups with at most 32 rows load a 32-row A box (the tensor core still multiplies 128 rows,
+// The small replicas of a shared expert are packed into common tiles (16-row slots, see the tile list
+// construction below).  Groups with at most 32 rows load a 32-row A box (the tensor core still multiplies 128 rows,
 // the extra rows are never stored), which keeps shared-memory fill traffic close to the weight
 // bytes in the weight-streaming regime.
 //
@@ -37,10 +38,12 @@ constexpr int BK = 64;
 constexpr int BN = 256;
 constexpr int kStages = 4;
 constexpr int kSmallRows = 32;
-constexpr int kMergeSlots = BM / kSmallRows;   // 32-row slots of a merged tile
+constexpr int kSlotRows = 16;                  // rows of one slot of a merged tile
+constexpr int kMergeSlots = BM / kSlotRows;    // slots of a merged tile
 constexpr int kMergeMaxRows = 64;              // replicas of a shared expert are merged when none has more rows
 constexpr int kABytes = BM * BK * 2;
 constexpr int kASmallBytes = kSmallRows * BK * 2;
+constexpr int kASlotBytes = kSlotRows * BK * 2;
 constexpr int kBBytes = BN * BK * 2;
 constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kPairStages = 6;
@@ -225,7 +228,7 @@ __device__ __forceinline__ float silu_mul(uint32_t g_bits, uint32_t u_bits) {
 template <int PHASE, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA_small,
-           const __grid_constant__ CUtensorMap tmB0, const __grid_constant__ CUtensorMap tmB1,
+           const __grid_constant__ CUtensorMap tmA_slot, const __grid_constant__ CUtensorMap tmB0, const __grid_constant__ CUtensorMap tmB1,
            const int4* __restrict__ work, const int2* __restrict__ slots, const int32_t* __restrict__ work_count,
            bf16* __restrict__ out, int ld_out, int n_out, int k_total, int* status) {
   EB_GRID_DEP_SYNC();
@@ -260,6 +263,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     prefetch_tmap(&tmA);
     if (!PAIR) prefetch_tmap(&tmA_small);
+    if (!PAIR) prefetch_tmap(&tmA_slot);
     prefetch_tmap(&tmB0);
     if (PHASE == 1) prefetch_tmap(&tmB1);
   }
@@ -289,47 +293,79 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
       uint32_t phase = 0;
       for (int w = w_first; w < n_work; w += w_step) {
         // x = first row, y = valid rows, z = weight matrix, w = n tile; y < 0 marks a merged tile:
-        // -y slots of 32 rows each, described by slots[x .. x - y)
+        // (-y & 15) slots of 16 rows each, or of 32 rows each if (-y & 16), described by slots[x ..)
         const int4 it = __ldg(work + w);
         const bool merged = !PAIR && it.y < 0;
-        const int n_slots = merged ? -it.y : 0;
+        const int n_slots = merged ? ((-it.y) & 15) : 0;
+        const bool big_slots = merged && ((-it.y) & 16);
         int slot_row[kMergeSlots];
 #pragma unroll
         for (int i = 0; i < kMergeSlots; ++i) slot_row[i] = (merged && i < n_slots) ? __ldg(slots + it.x + i).x : 0;
         const bool small = !PAIR && !merged && it.y <= kSmallRows;
         const uint32_t tx = PAIR ? 2u * kPairStageBytes
-                                 : (uint32_t)((merged ? n_slots * kASmallBytes : small ? kASmallBytes : kABytes) + kBBytes);
-        for (int kb = 0; kb < num_kb; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, s_abort, status)) goto done;
-          const uint32_t sa = base + stage * SB, sb = sa + kABytes;
-          if (PAIR) {
+                                 : (uint32_t)((merged ? n_slots * (big_slots ? kASmallBytes : kASlotBytes) : small ? kASmallBytes : kABytes) + kBBytes);
+        // One specialised k loop per tile kind, so the issuing thread does the minimum between a stage
+        // becoming free and its copies being in flight (that delay comes straight off the prefetch depth).
+#define EB_STAGE_BEGIN()                                                              \
+  if (!mbar_wait(empty_bar(stage), phase ^ 1u, s_abort, status)) goto done;           \
+  const uint32_t sa = base + stage * SB, sb = sa + kABytes;
+#define EB_STAGE_END()      \
+  if (++stage == NS) {      \
+    stage = 0;              \
+    phase ^= 1u;            \
+  }
+#define EB_LOAD_B_SINGLE()                                                                        \
+  if (PHASE == 1) {                                                                               \
+    tma_load_3d(sb, &tmB0, kb * BK, it.w * 128, it.z, full_bar(stage));                           \
+    tma_load_3d(sb + kBBytes / 2, &tmB1, kb * BK, it.w * 128, it.z, full_bar(stage));             \
+  } else {                                                                                        \
+    tma_load_3d(sb, &tmB0, kb * BK, it.w * BN, it.z, full_bar(stage));                            \
+  }
+        if (PAIR) {
+          const CUtensorMap* bmap = (PHASE == 1 && rank == 1) ? &tmB1 : &tmB0;
+          const int brow = PHASE == 1 ? it.w * 128 : it.w * BN + (int)rank * 128;
+          for (int kb = 0; kb < num_kb; ++kb) {
+            EB_STAGE_BEGIN();
             // both CTAs' copies are counted on the leader's barrier; the leader announces the total
             const uint32_t fb = map_to_cta(full_bar(stage), 0);
             if (rank == 0) mbar_expect_tx(full_bar(stage), tx);
             tma_pair_load_2d(sa, &tmA, kb * BK, it.x + (int)rank * BM, fb);
-            if (PHASE == 1) tma_pair_load_3d(sb, rank == 0 ? &tmB0 : &tmB1, kb * BK, it.w * 128, it.z, fb);
-            else tma_pair_load_3d(sb, &tmB0, kb * BK, it.w * BN + (int)rank * 128, it.z, fb);
-          } else {
-            mbar_expect_tx(full_bar(stage), tx);
-            if (merged) {
-#pragma unroll
-              for (int i = 0; i < kMergeSlots; ++i)
-                if (i < n_slots) tma_load_2d(sa + i * kASmallBytes, &tmA_small, kb * BK, slot_row[i], full_bar(stage));
-            } else {
-              tma_load_2d(sa, small ? &tmA_small : &tmA, kb * BK, it.x, full_bar(stage));
-            }
-            if (PHASE == 1) {
-              tma_load_3d(sb, &tmB0, kb * BK, it.w * 128, it.z, full_bar(stage));
-              tma_load_3d(sb + kBBytes / 2, &tmB1, kb * BK, it.w * 128, it.z, full_bar(stage));
-            } else {
-              tma_load_3d(sb, &tmB0, kb * BK, it.w * BN, it.z, full_bar(stage));
-            }
+            tma_pair_load_3d(sb, bmap, kb * BK, brow, it.z, fb);
+            EB_STAGE_END();
           }
-          if (++stage == NS) {
-            stage = 0;
-            phase ^= 1u;
+        } else if (!merged) {
+          const CUtensorMap* amap = small ? &tmA_small : &tmA;
+          for (int kb = 0; kb < num_kb; ++kb) {
+            EB_STAGE_BEGIN();
+            mbar_expect_tx(full_bar(stage), tx);
+            tma_load_2d(sa, amap, kb * BK, it.x, full_bar(stage));
+            EB_LOAD_B_SINGLE();
+            EB_STAGE_END();
+          }
+        } else if (big_slots) {
+          for (int kb = 0; kb < num_kb; ++kb) {
+            EB_STAGE_BEGIN();
+            mbar_expect_tx(full_bar(stage), tx);
+#pragma unroll
+            for (int i = 0; i < BM / kSmallRows; ++i)
+              if (i < n_slots) tma_load_2d(sa + i * kASmallBytes, &tmA_small, kb * BK, slot_row[i], full_bar(stage));
+            EB_LOAD_B_SINGLE();
+            EB_STAGE_END();
+          }
+        } else {
+          for (int kb = 0; kb < num_kb; ++kb) {
+            EB_STAGE_BEGIN();
+            mbar_expect_tx(full_bar(stage), tx);
+#pragma unroll
+            for (int i = 0; i < kMergeSlots; ++i)
+              if (i < n_slots) tma_load_2d(sa + i * kASlotBytes, &tmA_slot, kb * BK, slot_row[i], full_bar(stage));
+            EB_LOAD_B_SINGLE();
+            EB_STAGE_END();
           }
         }
+#undef EB_STAGE_BEGIN
+#undef EB_STAGE_END
+#undef EB_LOAD_B_SINGLE
       }
     }
   } else if (warp == 1) {
@@ -379,12 +415,16 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
       bool row_ok = r < it.y;
       int row_g = it.x + r;                     // row in the permuted order
       if (!PAIR && it.y < 0) {
-        // merged tile: epilogue warp q owns slot q (32 rows of one replica group)
+        // merged tile: epilogue warp q owns slot q (32-row slots) or slots 2q and 2q+1 (16-row slots)
         row_ok = false;
-        if (q < -it.y) {
-          const int2 sl = __ldg(slots + it.x + q);
-          row_g = sl.x + lane;
-          row_ok = lane < sl.y;
+        const int v = -it.y;
+        const bool big = v & 16;
+        const int slot = big ? q : 2 * q + (lane >> 4);
+        const int local_row = big ? lane : (lane & 15);
+        if (slot < (v & 15)) {
+          const int2 sl = __ldg(slots + it.x + slot);
+          row_g = sl.x + local_row;
+          row_ok = local_row < sl.y;
         }
       }
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + as * BN;
@@ -514,7 +554,7 @@ __device__ __forceinline__ int group_at(const ModelParams& mp, const int* dev_of
 }
 
 // The D replicas of a shared expert, when all are small, are packed into common 128-row tiles: the rows
-// of each replica are cut into chunks of 32 (one TMA box, one epilogue warp), four chunks per tile, so
+// of each replica are cut into chunks of 16 (one TMA box, half an epilogue warp), eight chunks per tile, so
 // the weight tile is fetched once for all of them.  `i` is a position of the processing order; returns
 // true if it belongs to such a merged class and gives the class's first position and chunk count.
 __device__ __forceinline__ bool merged_class(const ModelParams& mp, const int* dev_off, int nl, int device, int i,
@@ -522,15 +562,18 @@ __device__ __forceinline__ bool merged_class(const ModelParams& mp, const int* d
   if (device >= 0 || mp.S == 0 || mp.D < 2 || i < nl * mp.E) return false;
   const int q = i - nl * mp.E;
   const int h = i - q % mp.D;   // position of the class's replica on device 0
-  int tot = 0, mx = 0;
+  int tot16 = 0, tot32 = 0, mx = 0;
   for (int d = 0; d < mp.D; ++d) {
     const int g = group_at(mp, dev_off, nl, device, 0, h + d);
     const int rows = group_off[g + 1] - group_off[g];
-    tot += (rows + kSmallRows - 1) / kSmallRows;
+    tot16 += (rows + kSlotRows - 1) / kSlotRows;
+    tot32 += (rows + kSmallRows - 1) / kSmallRows;
     mx = rows > mx ? rows : mx;
   }
   *head = h;
-  *chunks = tot;
+  // 16-row slots (eight per tile) when every replica fits one, else 32-row slots (four per tile);
+  // bit 30 of *chunks marks the larger slots
+  *chunks = mx <= kSlotRows ? tot16 : (tot32 | (1 << 30));
   return mx <= kMergeMaxRows;
 }
 
@@ -563,7 +606,8 @@ plan_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t
       pgroup[i] = g;
       pchunks[i] = -1;
       if (merged_class(mp, s_dev_off, nl, device, i, group_off, &head, &chunks)) {
-        v = i == head ? (chunks + kMergeSlots - 1) / kMergeSlots : 0;   // the class's tiles sit at its first position
+        const int per_tile = (chunks >> 30) ? BM / kSmallRows : kMergeSlots;
+        v = i == head ? ((chunks & 0xffff) + per_tile - 1) / per_tile : 0;   // the class's tiles sit at its first position
         pchunks[i] = chunks;
       } else if (pair_mode && group_uses_pairs(rows)) {
         v = (long long)((rows + 2 * BM - 1) / (2 * BM)) << 32;
@@ -649,24 +693,28 @@ fill_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t
     const int n = rem / t_g, m = rem % t_g;
     const int g = pgroup[gi];
     int4 it;
-    const int head = gi, chunks = pchunks[gi];   // only the first position of a merged class owns tiles
-    if (!pair && chunks >= 0) {
-      // tile m of a merged class holds chunks 4m .. 4m+3 of the class (replicas in device order)
+    const int head = gi, chunks_raw = pchunks[gi];   // only the first position of a merged class owns tiles
+    if (!pair && chunks_raw >= 0) {
+      // tile m of a merged class holds the next 8 (16-row) or 4 (32-row) chunks of the class, replicas in
+      // device order
+      const bool big = (chunks_raw >> 30) & 1;
+      const int chunks = chunks_raw & 0xffff;
+      const int slot_rows = big ? kSmallRows : kSlotRows, per_tile = BM / slot_rows;
       const int base = kMergeSlots * (pref[gi] + m);
-      const int first = kMergeSlots * m, n_here = min(kMergeSlots, chunks - first);
+      const int first = per_tile * m, n_here = min(per_tile, chunks - first);
       if (list == 0 && n == 0) {
         int c = 0;   // chunks before the current replica
         for (int d = 0; d < mp.D; ++d) {
           const int gd = pgroup[head + d];
           const int r0 = group_off[gd], rows = group_off[gd + 1] - r0;
-          const int nc = (rows + kSmallRows - 1) / kSmallRows;
+          const int nc = (rows + slot_rows - 1) / slot_rows;
           for (int k = 0; k < nc; ++k, ++c)
             if (c >= first && c < first + n_here)
-              slots[base + c - first] = make_int2(r0 + k * kSmallRows, min(kSmallRows, rows - k * kSmallRows));
+              slots[base + c - first] = make_int2(r0 + k * slot_rows, min(slot_rows, rows - k * slot_rows));
         }
       }
       it.x = base;
-      it.y = -n_here;
+      it.y = -(n_here | (big ? 16 : 0));
     } else {
       const int row0 = group_off[g] + m * tile_rows;
       it.x = row0;
@@ -714,7 +762,8 @@ bool make_map(CUtensorMap* m, const void* ptr, uint64_t d0, uint64_t d1, uint64_
 
 template <int PHASE, bool PAIR>
 cudaError_t launch_ffn(eb_ctx* c, cudaStream_t st, const CUtensorMap& tA, const CUtensorMap& tAs, const CUtensorMap& tB0,
-                       const CUtensorMap& tB1, const int4* work, bf16* out, int ld_out, int n_out, int k_total) {
+                       const CUtensorMap& tB1, const int4* work, bf16* out, int ld_out, int n_out, int k_total,
+                       const CUtensorMap& tAslot) {
   const int2* slots = c->slots;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(PAIR ? c->pair_grid : c->num_sms);
@@ -732,7 +781,7 @@ cudaError_t launch_ffn(eb_ctx* c, cudaStream_t st, const CUtensorMap& tA, const 
   cfg.numAttrs = 2;
   const int32_t* wc = c->work_count;
   ++g_ebi_launches;
-  return cudaLaunchKernelEx(&cfg, ffn_kernel<PHASE, PAIR>, tA, tAs, tB0, tB1, work, slots, wc, out, ld_out, n_out, k_total,
+  return cudaLaunchKernelEx(&cfg, ffn_kernel<PHASE, PAIR>, tA, tAs, tAslot, tB0, tB1, work, slots, wc, out, ld_out, n_out, k_total,
                             c->d_status);
 }
 
@@ -791,9 +840,10 @@ eb_status ebi_ffn_run(eb_ctx* c, cudaStream_t st, const void* xp, const int32_t*
   if (!c->ws) return ebi_fail(c, EB_ERR_WORKSPACE, "no workspace set");
   const eb_config& g = c->cfg;
   const int rows = ebi_rows_cap(c);
-  CUtensorMap tm_x, tm_xs, tm_a, tm_as;
+  CUtensorMap tm_x, tm_xs, tm_xl, tm_a, tm_as, tm_al;
   if (!make_map(&tm_x, xp, g.H, rows, 0, BK, BM) || !make_map(&tm_xs, xp, g.H, rows, 0, BK, kSmallRows) ||
-      !make_map(&tm_a, c->act, g.I, rows, 0, BK, BM) || !make_map(&tm_as, c->act, g.I, rows, 0, BK, kSmallRows))
+      !make_map(&tm_xl, xp, g.H, rows, 0, BK, kSlotRows) || !make_map(&tm_a, c->act, g.I, rows, 0, BK, BM) ||
+      !make_map(&tm_as, c->act, g.I, rows, 0, BK, kSmallRows) || !make_map(&tm_al, c->act, g.I, rows, 0, BK, kSlotRows))
     return ebi_fail(c, EB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the activations");
   const int nt1 = (g.I + 127) / 128, nt2 = (g.H + BN - 1) / BN;
   // CTA pairs only pay for groups of more than 128 rows; skip their launches when the permutation that
@@ -815,19 +865,19 @@ eb_status ebi_ffn_run(eb_ctx* c, cudaStream_t st, const void* xp, const int32_t*
   cudaError_t e = cudaSuccess;
   if (pairs) {
     KernelTimer timer(c, EBK_FFN_GATEUP_PAIR, st);
-    e = launch_ffn<1, true>(c, st, tm_x, tm_xs, c->tm_gate, c->tm_up, c->work1p, c->act, g.I, g.I, g.H);
+    e = launch_ffn<1, true>(c, st, tm_x, tm_xs, c->tm_gate, c->tm_up, c->work1p, c->act, g.I, g.I, g.H, tm_xl);
   }
   if (e == cudaSuccess) {
     KernelTimer timer(c, EBK_FFN_GATEUP, st);
-    e = launch_ffn<1, false>(c, st, tm_x, tm_xs, c->tm_gate, c->tm_up, c->work1, c->act, g.I, g.I, g.H);
+    e = launch_ffn<1, false>(c, st, tm_x, tm_xs, c->tm_gate, c->tm_up, c->work1, c->act, g.I, g.I, g.H, tm_xl);
   }
   if (e == cudaSuccess && pairs) {
     KernelTimer timer(c, EBK_FFN_DOWN_PAIR, st);
-    e = launch_ffn<2, true>(c, st, tm_a, tm_as, c->tm_down_half, c->tm_down_half, c->work2p, (bf16*)yp, g.H, g.H, g.I);
+    e = launch_ffn<2, true>(c, st, tm_a, tm_as, c->tm_down_half, c->tm_down_half, c->work2p, (bf16*)yp, g.H, g.H, g.I, tm_al);
   }
   if (e == cudaSuccess) {
     KernelTimer timer(c, EBK_FFN_DOWN, st);
-    e = launch_ffn<2, false>(c, st, tm_a, tm_as, c->tm_down, c->tm_down, c->work2, (bf16*)yp, g.H, g.H, g.I);
+    e = launch_ffn<2, false>(c, st, tm_a, tm_as, c->tm_down, c->tm_down, c->work2, (bf16*)yp, g.H, g.H, g.I, tm_al);
   }
   if (e != cudaSuccess) return ebi_check_cuda(c, e, "expert_ffn launch");
   EB_LAUNCH_CHECK(c, "expert_ffn");

@@ -87,7 +87,7 @@ struct eb_ctx {
   int4* work2 = nullptr;           // down tile list
   int4* work1p = nullptr;          // gate/up tile list of the CTA-pair kernel
   int4* work2p = nullptr;          // down tile list of the CTA-pair kernel
-  int2* slots = nullptr;           // [4 * max_mtiles] (first row, rows) of the 32-row slots of merged tiles
+  int2* slots = nullptr;           // [8 * max_mtiles] (first row, rows) of the 16-row slots of merged tiles
   bf16* act = nullptr;             // [R_cap][I]
   int32_t max_chunks = 0, max_mtiles = 0, max_work1 = 0, max_work2 = 0, max_work1p = 0, max_work2p = 0;
 
