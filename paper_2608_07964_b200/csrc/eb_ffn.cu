@@ -9,8 +9,9 @@
 // contiguous K-major operand, so one tcgen05.mma feeds both and the epilogue fuses SiLU * up.
 //
 // Per CTA (one per SM): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
-// warps 2..5 = epilogue (TMEM -> registers -> bf16 -> global).  Shared memory holds a 4-stage
-// ring of {A 128x64, B 256x64} bf16 tiles in the 128-byte swizzled K-major layout; TMEM holds two
+// warps 2..5 = epilogue (TMEM -> registers -> bf16 -> global).  Shared memory holds a 4-stage ring of
+// A tiles (128x64) and a 5-stage ring of B tiles (256x64), bf16 in the 128-byte swizzled K-major
+// layout, each ring with its own barriers so the weight copies run one k-block further ahead; TMEM holds two
 // 128x256 fp32 accumulators so the epilogue of tile i overlaps the MMAs of tile i+1.
 // Tiles of one group are ordered weight-tile-major, so CTAs working side by side share the
 // weight tile in L2 and every weight byte leaves HBM once per group; the replicas of a shared expert on
@@ -36,7 +37,8 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;
 constexpr int BN = 256;
-constexpr int kStages = 4;
+constexpr int kStagesA = 4;   // single-CTA kernel: ring of A tiles (token rows)
+constexpr int kStagesB = 5;   // single-CTA kernel: ring of B tiles (weights): one deeper, they come from DRAM
 constexpr int kSmallRows = 32;
 constexpr int kSlotRows = 16;                  // rows of one slot of a merged tile
 constexpr int kMergeSlots = BM / kSlotRows;    // slots of a merged tile
@@ -46,12 +48,15 @@ constexpr int kASmallBytes = kSmallRows * BK * 2;
 constexpr int kASlotBytes = kSlotRows * BK * 2;
 constexpr int kBBytes = BN * BK * 2;
 constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kPairStages = 6;
+constexpr int kPairStages = 7;
 constexpr int kPairStageBytes = kABytes + kBBytes / 2;   // per CTA of a pair: own A rows + half of B
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 512;
-constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-static_assert(kPairStages * kPairStageBytes == kStages * kStageBytes, "both variants use the same ring size");
+constexpr size_t kSingleRingBytes = (size_t)kStagesA * kABytes + (size_t)kStagesB * kBBytes;
+constexpr size_t kPairRingBytes = (size_t)kPairStages * kPairStageBytes;
+constexpr size_t kRingBytes = kSingleRingBytes > kPairRingBytes ? kSingleRingBytes : kPairRingBytes;
+constexpr size_t kSmemBytes = kRingBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 constexpr long long kSpinLimitCycles = 4000000000LL;
 
 // ---- PTX wrappers ----------------------------------------------------------------------------
@@ -232,28 +237,39 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
            const int4* __restrict__ work, const int2* __restrict__ slots, const int32_t* __restrict__ work_count,
            bf16* __restrict__ out, int ld_out, int n_out, int k_total, int* status) {
   EB_GRID_DEP_SYNC();
-  constexpr int NS = PAIR ? kPairStages : kStages;
-  constexpr int SB = PAIR ? kPairStageBytes : kStageBytes;
+  // Pair kernel: one ring of kPairStages stages holding {A rows, half of B}.  Single-CTA kernel: two rings,
+  // kStagesA stages of A and kStagesB stages of B, each with its own full/empty barriers, so the weight
+  // copies (DRAM latency) run one k-block further ahead than shared memory would allow with joint stages.
+  constexpr int NA = PAIR ? kPairStages : kStagesA;
+  constexpr int NB = PAIR ? 0 : kStagesB;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - raw);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)NS * SB);
-  // barrier indices: full[0..NS), empty[NS..2NS), tmem_full[2NS, 2NS+2), tmem_empty[2NS+2, 2NS+4)
-  const uint32_t bar0 = base + NS * SB;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kRingBytes);
+  const uint32_t bar0 = base + (uint32_t)kRingBytes;
+  auto a_addr = [&](int s) { return PAIR ? base + s * kPairStageBytes : base + s * kABytes; };
+  auto b_addr = [&](int s) { return PAIR ? base + s * kPairStageBytes + kABytes : base + kStagesA * kABytes + s * kBBytes; };
+  // barriers: full_a[NA], empty_a[NA], full_b[NB], empty_b[NB], tmem_full[2], tmem_empty[2]
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (NS + s); };
-  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * NS + a); };
-  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * NS + 2 + a); };
-  volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(bars + 2 * NS + 4);
-  volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 2 * NS + 5);
+  auto empty_bar = [&](int s) { return bar0 + 8u * (NA + s); };
+  auto fullb_bar = [&](int s) { return bar0 + 8u * (2 * NA + s); };
+  auto emptyb_bar = [&](int s) { return bar0 + 8u * (2 * NA + NB + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * NA + 2 * NB + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * NA + 2 * NB + 2 + a); };
+  volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(bars + 2 * NA + 2 * NB + 4);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 2 * NA + 2 * NB + 5);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = PAIR ? cluster_ctarank() : 0u;   // CTA 0 of a pair is the leader
   if (threadIdx.x == 0) {
-    for (int s = 0; s < NS; ++s) {
+    for (int s = 0; s < NA; ++s) {
       mbar_init(full_bar(s), 1);    // producer's arrive + all bytes of the stage (pair: of both CTAs, leader only)
       mbar_init(empty_bar(s), 1);   // one tcgen05.commit
+    }
+    for (int s = 0; s < NB; ++s) {
+      mbar_init(fullb_bar(s), 1);
+      mbar_init(emptyb_bar(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);                // one tcgen05.commit
@@ -289,8 +305,8 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
+      int stage = 0, stage_b = 0;
+      uint32_t phase = 0, phase_b = 0;
       for (int w = w_first; w < n_work; w += w_step) {
         // x = first row, y = valid rows, z = weight matrix, w = n tile; y < 0 marks a merged tile:
         // (-y & 15) slots of 16 rows each, or of 32 rows each if (-y & 16), described by slots[x ..)
@@ -302,77 +318,87 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
 #pragma unroll
         for (int i = 0; i < kMergeSlots; ++i) slot_row[i] = (merged && i < n_slots) ? __ldg(slots + it.x + i).x : 0;
         const bool small = !PAIR && !merged && it.y <= kSmallRows;
-        const uint32_t tx = PAIR ? 2u * kPairStageBytes
-                                 : (uint32_t)((merged ? n_slots * (big_slots ? kASmallBytes : kASlotBytes) : small ? kASmallBytes : kABytes) + kBBytes);
+        const uint32_t tx_a = (uint32_t)(merged ? n_slots * (big_slots ? kASmallBytes : kASlotBytes) : small ? kASmallBytes : kABytes);
         // One specialised k loop per tile kind, so the issuing thread does the minimum between a stage
         // becoming free and its copies being in flight (that delay comes straight off the prefetch depth).
-#define EB_STAGE_BEGIN()                                                              \
+        // Single-CTA kernel: the weight copy of a k-block goes out first (it has the DRAM latency), then
+        // the A copy once its own ring has room.
+#define EB_B_STAGE()                                                                              \
+  if (!mbar_wait(emptyb_bar(stage_b), phase_b ^ 1u, s_abort, status)) goto done;                  \
+  {                                                                                               \
+    const uint32_t sb = b_addr(stage_b);                                                          \
+    mbar_expect_tx(fullb_bar(stage_b), kBBytes);                                                  \
+    if (PHASE == 1) {                                                                             \
+      tma_load_3d(sb, &tmB0, kb * BK, it.w * 128, it.z, fullb_bar(stage_b));                      \
+      tma_load_3d(sb + kBBytes / 2, &tmB1, kb * BK, it.w * 128, it.z, fullb_bar(stage_b));        \
+    } else {                                                                                      \
+      tma_load_3d(sb, &tmB0, kb * BK, it.w * BN, it.z, fullb_bar(stage_b));                       \
+    }                                                                                             \
+    if (++stage_b == kStagesB) {                                                                  \
+      stage_b = 0;                                                                                \
+      phase_b ^= 1u;                                                                              \
+    }                                                                                             \
+  }
+#define EB_A_STAGE_BEGIN()                                                            \
   if (!mbar_wait(empty_bar(stage), phase ^ 1u, s_abort, status)) goto done;           \
-  const uint32_t sa = base + stage * SB, sb = sa + kABytes;
-#define EB_STAGE_END()      \
-  if (++stage == NS) {      \
+  const uint32_t sa = a_addr(stage);
+#define EB_A_STAGE_END()    \
+  if (++stage == NA) {      \
     stage = 0;              \
     phase ^= 1u;            \
-  }
-#define EB_LOAD_B_SINGLE()                                                                        \
-  if (PHASE == 1) {                                                                               \
-    tma_load_3d(sb, &tmB0, kb * BK, it.w * 128, it.z, full_bar(stage));                           \
-    tma_load_3d(sb + kBBytes / 2, &tmB1, kb * BK, it.w * 128, it.z, full_bar(stage));             \
-  } else {                                                                                        \
-    tma_load_3d(sb, &tmB0, kb * BK, it.w * BN, it.z, full_bar(stage));                            \
   }
         if (PAIR) {
           const CUtensorMap* bmap = (PHASE == 1 && rank == 1) ? &tmB1 : &tmB0;
           const int brow = PHASE == 1 ? it.w * 128 : it.w * BN + (int)rank * 128;
           for (int kb = 0; kb < num_kb; ++kb) {
-            EB_STAGE_BEGIN();
+            EB_A_STAGE_BEGIN();
             // both CTAs' copies are counted on the leader's barrier; the leader announces the total
             const uint32_t fb = map_to_cta(full_bar(stage), 0);
-            if (rank == 0) mbar_expect_tx(full_bar(stage), tx);
+            if (rank == 0) mbar_expect_tx(full_bar(stage), 2u * kPairStageBytes);
             tma_pair_load_2d(sa, &tmA, kb * BK, it.x + (int)rank * BM, fb);
-            tma_pair_load_3d(sb, bmap, kb * BK, brow, it.z, fb);
-            EB_STAGE_END();
+            tma_pair_load_3d(b_addr(stage), bmap, kb * BK, brow, it.z, fb);
+            EB_A_STAGE_END();
           }
         } else if (!merged) {
           const CUtensorMap* amap = small ? &tmA_small : &tmA;
           for (int kb = 0; kb < num_kb; ++kb) {
-            EB_STAGE_BEGIN();
-            mbar_expect_tx(full_bar(stage), tx);
+            EB_B_STAGE();
+            EB_A_STAGE_BEGIN();
+            mbar_expect_tx(full_bar(stage), tx_a);
             tma_load_2d(sa, amap, kb * BK, it.x, full_bar(stage));
-            EB_LOAD_B_SINGLE();
-            EB_STAGE_END();
+            EB_A_STAGE_END();
           }
         } else if (big_slots) {
           for (int kb = 0; kb < num_kb; ++kb) {
-            EB_STAGE_BEGIN();
-            mbar_expect_tx(full_bar(stage), tx);
+            EB_B_STAGE();
+            EB_A_STAGE_BEGIN();
+            mbar_expect_tx(full_bar(stage), tx_a);
 #pragma unroll
             for (int i = 0; i < BM / kSmallRows; ++i)
               if (i < n_slots) tma_load_2d(sa + i * kASmallBytes, &tmA_small, kb * BK, slot_row[i], full_bar(stage));
-            EB_LOAD_B_SINGLE();
-            EB_STAGE_END();
+            EB_A_STAGE_END();
           }
         } else {
           for (int kb = 0; kb < num_kb; ++kb) {
-            EB_STAGE_BEGIN();
-            mbar_expect_tx(full_bar(stage), tx);
+            EB_B_STAGE();
+            EB_A_STAGE_BEGIN();
+            mbar_expect_tx(full_bar(stage), tx_a);
 #pragma unroll
             for (int i = 0; i < kMergeSlots; ++i)
               if (i < n_slots) tma_load_2d(sa + i * kASlotBytes, &tmA_slot, kb * BK, slot_row[i], full_bar(stage));
-            EB_LOAD_B_SINGLE();
-            EB_STAGE_END();
+            EB_A_STAGE_END();
           }
         }
-#undef EB_STAGE_BEGIN
-#undef EB_STAGE_END
-#undef EB_LOAD_B_SINGLE
+#undef EB_B_STAGE
+#undef EB_A_STAGE_BEGIN
+#undef EB_A_STAGE_END
       }
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer (pair: leader CTA only) ----------------
     if (lane == 0 && rank == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
+      int stage = 0, stage_b = 0;
+      uint32_t phase = 0, phase_b = 0;
       int local = 0;
       for (int w = w_first; w < n_work; w += w_step, ++local) {
         const int as = local & 1;
@@ -382,17 +408,26 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
         const uint32_t d_tmem = tmem_base + as * BN;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, s_abort, status)) goto done;
+          if (!PAIR && !mbar_wait(fullb_bar(stage_b), phase_b, s_abort, status)) goto done;
           tc_fence_after();
-          const uint32_t sa = base + stage * SB, sb = sa + kABytes;
-          const uint64_t da = smem_desc(sa), db = smem_desc(sb);
+          const uint64_t da = smem_desc(a_addr(stage)), db = smem_desc(b_addr(PAIR ? stage : stage_b));
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k) {
             if (PAIR) umma_pair_bf16(d_tmem, da + 2 * k, db + 2 * k, kIdescPair, (kb | k) != 0 ? 1u : 0u);
             else umma_bf16(d_tmem, da + 2 * k, db + 2 * k, kIdesc, (kb | k) != 0 ? 1u : 0u);
           }
-          // smem stage reusable (in both CTAs of a pair) once these MMAs have read it
-          if (PAIR) umma_pair_commit(empty_bar(stage)); else umma_commit(empty_bar(stage));
-          if (++stage == NS) {
+          // the stages are reusable (in both CTAs of a pair) once these MMAs have read them
+          if (PAIR) {
+            umma_pair_commit(empty_bar(stage));
+          } else {
+            umma_commit(empty_bar(stage));
+            umma_commit(emptyb_bar(stage_b));
+            if (++stage_b == kStagesB) {
+              stage_b = 0;
+              phase_b ^= 1u;
+            }
+          }
+          if (++stage == NA) {
             stage = 0;
             phase ^= 1u;
           }
