@@ -437,3 +437,25 @@ def test_c5_sweep_point_full_step():
     # the most skewed point of the sweep with the largest micro-batch count
     wl = synth.workload_c5(16, 128, 1.5)
     _full_step(Hn.make_case(wl), Hn.WeightStore(wl), wl.m)
+
+
+def test_schedule_large_pools_split_over_blocks():
+    """Pools of 12 to 16 members: the MaxUtil enumeration runs on several blocks; ties are frequent with
+    these small loads, so the total order is exercised across block boundaries."""
+    B = _binding()
+    rng = np.random.default_rng(777)
+    wl = _small(D=4)
+    step = B.from_workload(wl, max_tokens=64)
+    for trial in range(10):
+        n_mb = 16
+        np_pool = [12, 13, 14, 15, 16][trial % 5]
+        members = sorted(rng.choice(n_mb, size=np_pool, replace=False).tolist())
+        pool = sum(1 << j for j in members)
+        m = int(rng.integers(max(1, np_pool - 5), np_pool))
+        loads = rng.integers(0, 4 if trial % 2 else 40, size=(n_mb, 4)).astype(np.int32)
+        dev_loads = torch.from_numpy(loads).cuda()
+        batch = B.Batch([0] * (n_mb + 1), [0] * n_mb, pool)
+        got = step.eb_schedule(batch, m, O.POLICY_MAXUTIL, to_host=True, mb_load=dev_loads)
+        ref = O.schedule(loads, pool, m, O.POLICY_MAXUTIL)
+        for k in ("run_mask", "defer_mask", "n_run", "joint_load", "util_num", "util_den"):
+            assert got[k] == ref[k], (trial, k, got[k], ref[k])
