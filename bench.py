@@ -40,8 +40,8 @@ UNIT = "tokens/s"
 # dram__bytes_write.sum over the algorithmic bytes of the captured launch.  The capture ran on the
 # 6-layer cut of the decode shape (profiles/ffn_c2small_ncu_full.md); traffic grows in proportion to
 # the weight bytes streamed, so a full launch is that ratio times its own algorithmic bytes.
-NCU_TRAFFIC_RATIO = {"c2": (1.488253e9 + 7.097344e6) / 1487011840.0,
-                     "c2small": (1.488253e9 + 7.097344e6) / 1487011840.0}
+NCU_TRAFFIC_RATIO = {"c2": (1.488622e9 + 7.138816e6) / 1487011840.0,
+                     "c2small": (1.488622e9 + 7.138816e6) / 1487011840.0}
 
 
 def measured_peaks():
