@@ -3,8 +3,10 @@
 // One warp per token.  Lane i holds logits i, i+32, ...  (E <= 256 -> at most 8 per lane).
 // K rounds of a warp arg-max under the order (value descending, index ascending) pick the
 // experts; the decision uses only comparisons on the raw fp32 logits, so it is exact.
-// Loads are integer counts accumulated per block in shared memory and flushed with integer
-// atomics (order independent).
+// Loads are integer counts added with integer atomics in global memory (order independent, hence
+// deterministic); a clearing kernel zeroes the rows of the micro-batches being routed first.  (Gathering
+// the counts per block in shared memory was tried: it needs several tokens per block to pay, and the lost
+// parallelism cost more than the atomics it saved.)
 #include "eb_internal.cuh"
 
 namespace {
