@@ -16,8 +16,8 @@
 // Tiles of one group are ordered weight-tile-major, so CTAs working side by side share the
 // weight tile in L2 and every weight byte leaves HBM once per group; the replicas of a shared expert on
 // the virtual devices are listed next to each other for the same reason.
-// The small replicas of a shared expert are packed into common tiles (16-row slots, see the tile list
-// construction below).  Groups with at most 32 rows load a 32-row A box (the tensor core still multiplies 128 rows,
+// The small replicas of a shared expert are packed into common tiles (16- or 32-row slots, see the tile
+// list construction below).  Groups with at most 32 rows load a 32-row A box (the tensor core still multiplies 128 rows,
 // the extra rows are never stored), which keeps shared-memory fill traffic close to the weight
 // bytes in the weight-streaming regime.
 //
@@ -25,7 +25,7 @@
 // owns a 256-row tile, each CTA loads its own 128 rows of A and one half of the weight tile (for
 // gate/up: CTA 0 the gate rows, CTA 1 the up rows), and the leader CTA issues tcgen05.mma
 // cta_group::2 (M = 256) that reads both halves.  A stage shrinks from 48 KB to 32 KB per CTA for the
-// same tensor-core time, so the ring deepens to 6 stages and L2 traffic per flop drops by a third -
+// same tensor-core time, so the ring deepens to 7 stages and L2 traffic per flop drops by a third -
 // that is what the tensor-bound regime needs.  No load is multicast; only tcgen05.commit is.
 //
 // Every wait on an mbarrier is bounded: on expiry the kernel records EB_ERR_TIMEOUT in the
@@ -47,7 +47,6 @@ constexpr int kABytes = BM * BK * 2;
 constexpr int kASmallBytes = kSmallRows * BK * 2;
 constexpr int kASlotBytes = kSlotRows * BK * 2;
 constexpr int kBBytes = BN * BK * 2;
-constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kPairStages = 7;
 constexpr int kPairStageBytes = kABytes + kBBytes / 2;   // per CTA of a pair: own A rows + half of B
 constexpr int kThreads = 192;
