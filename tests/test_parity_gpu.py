@@ -459,3 +459,38 @@ def test_schedule_large_pools_split_over_blocks():
         ref = O.schedule(loads, pool, m, O.POLICY_MAXUTIL)
         for k in ("run_mask", "defer_mask", "n_run", "joint_load", "util_num", "util_den"):
             assert got[k] == ref[k], (trial, k, got[k], ref[k])
+
+
+# ----------------------------------------------------------------------------------- randomised shapes
+def test_random_shapes_front_end_bit_exact():
+    """Routing, scheduling and permutation on 120 random shapes (experts, top-k, shared experts, devices,
+    micro-batch sizes, layers, pool, m, policy, mapping) against the oracle, bit for bit."""
+    rng = np.random.default_rng(2026)
+    for trial in range(120):
+        E = int(rng.integers(1, 40))
+        K = int(rng.integers(1, min(E, 8) + 1))
+        S = int(rng.integers(0, 4))
+        D = int(rng.integers(1, 9))
+        N = int(rng.integers(1, 9))
+        L = int(rng.integers(1, 6))
+        tokens = [int(v) for v in rng.integers(0, 70, size=N)]
+        if sum(tokens) == 0:
+            tokens[0] = 3
+        layers = [int(v) for v in rng.integers(0, L, size=N)]
+        pool = int(rng.integers(0, 1 << N))
+        m = int(rng.integers(1, N + 1))
+        policy = int(rng.integers(0, 4))
+        wl = synth.Workload(name=f"rnd{trial}", L=L, E=E, K=K, S=S, H=64, I=64, D=D,
+                            mapping=["mod", "contiguous"][trial % 2], N=N, T=8, zipf_s=float(rng.uniform(0, 1.5)),
+                            renorm_topk=trial % 3 != 0, seed=1000 + trial)
+        case = Hn.make_case(wl, tokens, layers)
+        _full_step(case, Hn.WeightStore(wl), m, policy, pool_mask=pool, check_ffn=(trial % 6 == 0))
+
+
+def test_other_policies_on_the_decode_and_fine_grained_shapes():
+    for name in ("c2", "c3"):
+        wl = synth.workload(name)
+        store = Hn.WeightStore(wl)
+        case = Hn.make_case(wl)
+        for pol in (O.POLICY_CUMUTIL, O.POLICY_DIFFPEAK, O.POLICY_ALL):
+            _full_step(case, store, wl.m, pol, check_ffn=False)
