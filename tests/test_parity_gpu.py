@@ -494,3 +494,23 @@ def test_other_policies_on_the_decode_and_fine_grained_shapes():
         case = Hn.make_case(wl)
         for pol in (O.POLICY_CUMUTIL, O.POLICY_DIFFPEAK, O.POLICY_ALL):
             _full_step(case, store, wl.m, pol, check_ffn=False)
+
+
+def test_random_expert_shapes_full_compare():
+    """Hidden and intermediate sizes that are multiples of 8 but of nothing larger, group sizes on both
+    sides of the 32-, 128- and 256-row tile boundaries, with and without shared experts: every expert output
+    and every aggregated output is compared."""
+    rng = np.random.default_rng(4242)
+    for trial in range(16):
+        H = 8 * int(rng.integers(1, 70))
+        I = 8 * int(rng.integers(1, 70))
+        E = int(rng.integers(2, 7))
+        K = int(rng.integers(1, min(E, 3) + 1))
+        S = int(rng.integers(0, 3))
+        D = int(rng.integers(1, 5))
+        N = int(rng.integers(1, 4))
+        tokens = [int(v) for v in rng.choice([1, 7, 33, 120, 129, 260, 400, 700], size=N)]
+        layers = [int(v) for v in rng.integers(0, 2, size=N)]
+        wl = synth.Workload(name=f"ffn{trial}", L=2, E=E, K=K, S=S, H=H, I=I, D=D, mapping="mod", N=N, T=8,
+                            zipf_s=float(rng.uniform(0, 2.0)), seed=500 + trial)
+        _full_step(Hn.make_case(wl, tokens, layers), Hn.WeightStore(wl), max(1, N - 1))
