@@ -120,7 +120,10 @@ typedef struct {
 
 /* Creates a context on the current CUDA device.  Allocates a few KB of device tables with
  * cudaMalloc.  Returns EB_ERR_UNSUPPORTED for shapes outside the limits, EB_ERR_INVALID_ARG
- * for a bad table, EB_ERR_CUDA if the device is not sm_100 or a CUDA call fails. */
+ * for a bad table, EB_ERR_CUDA if the device is not sm_100 or a CUDA call fails.  Every later
+ * call on the context must be made with that device current (EB_ERR_INVALID_ARG otherwise).  A
+ * context is not thread safe: calls on one context are made by one thread at a time; different
+ * contexts may be used from different threads. */
 eb_status eb_create(const eb_config* cfg, eb_ctx** out);
 eb_status eb_destroy(eb_ctx* ctx);
 

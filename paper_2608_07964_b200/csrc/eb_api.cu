@@ -6,9 +6,9 @@
 
 #include "eb_internal.cuh"
 
-unsigned long long g_ebi_launches = 0;
+std::atomic<unsigned long long> g_ebi_launches{0};
 
-extern "C" uint64_t eb_launch_count(void) { return g_ebi_launches; }
+extern "C" uint64_t eb_launch_count(void) { return g_ebi_launches.load(); }
 
 int32_t ebi_rows_cap(const eb_ctx* c) { return c->cfg.max_tokens * (c->cfg.K + c->cfg.S); }
 int32_t ebi_groups_cap(const eb_ctx* c) { return EB_MAX_MB * (c->cfg.E + c->cfg.D * c->cfg.S); }
@@ -24,7 +24,16 @@ eb_status ebi_check_cuda(eb_ctx* c, cudaError_t e, const char* what) {
   return ebi_fail(c, EB_ERR_CUDA, m);
 }
 
+eb_status ebi_check_device(eb_ctx* c) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return ebi_fail(c, EB_ERR_CUDA, "cudaGetDevice failed");
+  if (dev != c->device) return ebi_fail(c, EB_ERR_INVALID_ARG, "the context was created on another device than the current one");
+  return EB_OK;
+}
+
 eb_status ebi_make_batch(eb_ctx* c, const eb_batch* b, BatchParams* out) {
+  eb_status ds = ebi_check_device(c);
+  if (ds != EB_OK) return ds;
   if (!b || !b->tok_off || !b->layer) return ebi_fail(c, EB_ERR_INVALID_ARG, "null batch");
   if (b->n_mb < 0 || b->n_mb > EB_MAX_MB) return ebi_fail(c, EB_ERR_UNSUPPORTED, "n_mb out of range");
   if (b->n_mb < 32 && (b->pool_mask >> b->n_mb) != 0)

@@ -5,6 +5,8 @@
 // in flight together), accumulates in fp32 in the
 // fixed order k = 0..K-1 then s = 0..S-1, and stores bf16 (round to nearest even).  Gather form
 // means no atomics and a result that does not depend on scheduling.
+#include <utility>
+
 #include "eb_internal.cuh"
 
 namespace {
@@ -59,17 +61,12 @@ combine_kernel(int n_tok, int H, int K, int team, const uint4* __restrict__ yp, 
 
 typedef void (*combine_fn)(int, int, int, int, const uint4*, const int32_t*, const float*, uint4*);
 
-template <int KS>
-struct Table {
-  static void fill(combine_fn* f) {
-    f[KS] = combine_kernel<KS>;
-    Table<KS - 1>::fill(f);
-  }
-};
-template <>
-struct Table<0> {
-  static void fill(combine_fn*) {}
-};
+// kernel for every slot count 1 .. kMaxSlots (entry 0 unused)
+template <int... Is>
+const combine_fn* combine_table(std::integer_sequence<int, Is...>) {
+  static const combine_fn table[] = {nullptr, combine_kernel<Is + 1>...};
+  return table;
+}
 
 }  // namespace
 
@@ -82,12 +79,7 @@ extern "C" eb_status eb_combine(eb_ctx* c, void* stream, const eb_batch* batch, 
   if (!d_res || !yp || !pos || !topk_w || !out) return ebi_fail(c, EB_ERR_INVALID_ARG, "null pointer");
   if (!ebi_aligned16(yp) || !ebi_aligned16(out)) return ebi_fail(c, EB_ERR_INVALID_ARG, "yp / out must be 16-byte aligned");
   if (bp.n_tok == 0) return EB_OK;
-  static combine_fn table[kMaxSlots + 1] = {};
-  static bool init = false;
-  if (!init) {
-    Table<kMaxSlots>::fill(table);
-    init = true;
-  }
+  const combine_fn* table = combine_table(std::make_integer_sequence<int, kMaxSlots>());
   cudaStream_t st = (cudaStream_t)stream;
   const int KS = c->cfg.K + c->cfg.S;
   KernelTimer timer(c, EBK_COMBINE, st);

@@ -768,14 +768,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
+  static const EncodeTiledFn fn = [] {
     void* p = nullptr;
     cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = (EncodeTiledFn)p;
-  }
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return (EncodeTiledFn)p;
+  }();
   return fn;
 }
 
@@ -828,6 +828,7 @@ eb_status ebi_selftest_wait(eb_ctx* c, cudaStream_t st, long long limit_cycles, 
 }
 
 eb_status ebi_ffn_bind(eb_ctx* c) {
+  if (eb_status ds = ebi_check_device(c)) return ds;
   const eb_config& g = c->cfg;
   const uint64_t nw = (uint64_t)g.L * (g.E + g.S);
   if (!make_map(&c->tm_gate, c->w_gate, g.H, g.I, nw, BK, 128) ||
@@ -869,6 +870,7 @@ eb_status ebi_ffn_bind(eb_ctx* c) {
 eb_status ebi_ffn_run(eb_ctx* c, cudaStream_t st, const void* xp, const int32_t* group_off, const int32_t* group_w,
                       const int32_t* step_meta, void* yp, int32_t device) {
   if (!xp || !group_off || !group_w || !step_meta || !yp) return ebi_fail(c, EB_ERR_INVALID_ARG, "null pointer");
+  if (eb_status ds = ebi_check_device(c)) return ds;
   if (!ebi_aligned16(xp) || !ebi_aligned16(yp)) return ebi_fail(c, EB_ERR_INVALID_ARG, "xp / yp must be 16-byte aligned");
   if (!c->w_gate) return ebi_fail(c, EB_ERR_INVALID_ARG, "weights not bound");
   if (!c->ws) return ebi_fail(c, EB_ERR_WORKSPACE, "no workspace set");

@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
 #include <string>
 #include <vector>
 
@@ -104,6 +105,8 @@ int32_t ebi_groups_cap(const eb_ctx* c);
 eb_status ebi_fail(eb_ctx* c, eb_status s, const std::string& msg);
 eb_status ebi_check_cuda(eb_ctx* c, cudaError_t e, const char* what);
 eb_status ebi_make_batch(eb_ctx* c, const eb_batch* b, BatchParams* out);
+// EB_OK if the calling thread's current device is the one the context was created on.
+eb_status ebi_check_device(eb_ctx* c);
 
 // Brackets a launch with events when timing is enabled.
 struct KernelTimer {
@@ -140,7 +143,7 @@ struct KernelTimer {
 #define EB_GRID_DEP_SYNC() asm volatile("griddepcontrol.wait;\n\tgriddepcontrol.launch_dependents;" ::: "memory")
 
 // Number of kernels this library has launched in the process (all contexts).
-extern unsigned long long g_ebi_launches;
+extern std::atomic<unsigned long long> g_ebi_launches;
 
 template <typename... KArgs, typename... Args>
 static inline cudaError_t ebi_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,

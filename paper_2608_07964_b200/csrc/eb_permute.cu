@@ -24,32 +24,6 @@ struct StepShape {
   int rank_of_mb[EB_MAX_MB];    // rank of the micro-batch's layer among active layers, -1 if not chosen
 };
 
-__device__ __forceinline__ StepShape step_shape(const BatchParams& bp, uint32_t run) {
-  StepShape s;
-  s.nl = 0;
-  // insertion of distinct layers in ascending order (n_mb <= 16)
-  for (int j = 0; j < bp.n_mb; ++j) {
-    if (!((run >> j) & 1u)) continue;
-    int l = bp.layer[j], p = 0;
-    bool dup = false;
-    for (int i = 0; i < s.nl; ++i) {
-      if (s.act_layer[i] == l) dup = true;
-      if (s.act_layer[i] < l) p = i + 1;
-    }
-    if (dup) continue;
-    for (int i = s.nl; i > p; --i) s.act_layer[i] = s.act_layer[i - 1];
-    s.act_layer[p] = l;
-    ++s.nl;
-  }
-  for (int j = 0; j < EB_MAX_MB; ++j) {
-    s.rank_of_mb[j] = -1;
-    if (j < bp.n_mb && ((run >> j) & 1u))
-      for (int i = 0; i < s.nl; ++i)
-        if (s.act_layer[i] == bp.layer[j]) s.rank_of_mb[j] = i;
-  }
-  return s;
-}
-
 // first token (local index) of micro-batch of T tokens whose home device is >= d
 __device__ __forceinline__ int home_start(int d, int T, int D) {
   if (T < (1 << 26)) return (int)(((unsigned)d * (unsigned)T + (unsigned)(D - 1)) / (unsigned)D);   // d <= 16: no overflow
@@ -61,8 +35,8 @@ __device__ __forceinline__ int home_device(int tl, int T, int D) {
   return (int)(((long long)tl * D) / T);
 }
 
-// Block-cooperative version of step_shape: threads 0..15 each place one micro-batch, the result lands in
-// shared memory.  Ends with a block barrier.
+// Active layers of a step and every micro-batch's rank among them: threads 0..15 each place one
+// micro-batch, the result lands in shared memory.  Ends with a block barrier.
 __device__ __forceinline__ void step_shape_block(const BatchParams& bp, uint32_t run, StepShape* out) {
   const int j = threadIdx.x;
   if (j < EB_MAX_MB) {
@@ -91,13 +65,6 @@ __device__ __forceinline__ void step_shape_block(const BatchParams& bp, uint32_t
 __device__ __forceinline__ int group_id(const int* dev_off, int S, int nl, int d, int lr, int local) {
   int n_d = dev_off[d + 1] - dev_off[d];
   return nl * (dev_off[d] + d * S) + lr * (n_d + S) + local;
-}
-
-// Copies the per-device expert offsets into shared memory (independent loads issued together) so the
-// group decoding below does not chase dependent global loads.  Ends with a block barrier.
-__device__ __forceinline__ void stage_dev_off(const ModelParams& mp, int* s_dev_off) {
-  if (threadIdx.x <= mp.D) s_dev_off[threadIdx.x] = mp.dev_off[threadIdx.x];
-  __syncthreads();
 }
 
 __device__ __forceinline__ int mb_of_chunk(const BatchParams& bp, int c) {
