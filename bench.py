@@ -5,8 +5,9 @@ combine) on seeded synthetic inputs shaped like the benchmark configurations.
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
 
 Prints ONE JSON line.  `value` is tokens of the chosen micro-batches per second with all inputs
-resident in HBM; `e2e` is the same through eb_step_host with pinned host buffers (host<->device
-copies inside the timed region).  With N > 1 (torchrun) every rank runs an independent replica
+resident in HBM; `e2e` is the same with pinned host buffers, every step copying its inputs in and its result
+out inside the timed region, two steps in flight (eb_step_host_submit / eb_step_host_wait;
+`e2e.one_step_at_a_time` is the blocking eb_step_host).  With N > 1 (torchrun) every rank runs an independent replica
 on its own seeded batch (no collective on the data path); rank 0 reports the aggregate.
 `--impl reference` times the CPU oracle on a bounded sample of the same workload.
 """
@@ -338,12 +339,34 @@ def run_ours(args, wl):
     run_host = lambda: step.eb_step_host(batch, m, h_logits, h_x, h_out)
     side = torch.cuda.Stream()      # a stream of its own: the legacy default stream adds implicit synchronisation
     side.wait_stream(torch.cuda.current_stream())
+    # the same with two steps in flight (eb_step_host_submit / eb_step_host_wait): the copies of one step overlap
+    # the kernels of the other; every step still copies its inputs in and its result out inside the timed region
+    depth = 2
+    h_outs = [torch.empty((T, wl.H), dtype=torch.bfloat16).pin_memory() for _ in range(depth)]
+
+    def run_pipelined(n):
+        for i in range(n):
+            s = i % depth
+            if i >= depth:
+                step.step_host_wait(s)
+            step.step_host_submit(s, batch, m, h_logits, h_x, h_outs[s])
+        for s in range(min(depth, n)):
+            step.step_host_wait(s)
+
     with torch.cuda.stream(side):
         for _ in range(max(args.warmup, 3)):
             run_host()
         barrier()
-        ms_e2e = timed(run_host, args.steps)
+        ms_e2e_blocking = timed(run_host, args.steps)
+        run_pipelined(max(args.warmup, 3))
+        barrier()
+        ms_e2e = timed(lambda: run_pipelined(args.steps), 1)
     barrier()
+    for h in h_outs:      # rows of deferred micro-batches are not written by a step
+        for j in range(wl.N):
+            if (sched["run_mask"] >> j) & 1:
+                a, b = wl.tok_off[j], wl.tok_off[j + 1]
+                assert torch.equal(h[a:b], h_out[a:b]), "pipelined host path disagrees with the blocking one"
 
     # ---- reductions over ranks
     ms_max, ms_e2e_max, tok_total = reduce_over_ranks(dist, red_device, ms, ms_e2e, float(tokens_run))
@@ -406,7 +429,8 @@ def run_ours(args, wl):
                 ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
                 data="synthetic", config=workload_config(wl), clocks=clocks,
                 e2e=dict(value=tok_total / (ms_e2e_max / args.steps / 1e3), unit=UNIT, h2d_bytes_per_step=h2d,
-                         d2h_bytes_per_step=d2h),
+                         d2h_bytes_per_step=d2h, mode="host buffers, 2 steps in flight (eb_step_host_submit/_wait)",
+                         one_step_at_a_time=tokens_run / (ms_e2e_blocking / args.steps / 1e3)),
                 gpu_launches=launches, roofline=roof, cpu_baseline=cpu,
                 tokens_per_step=tok_total, run_mask=sched["run_mask"], device_status=status, idle=idle, detail=extra)
     print(json.dumps(line))

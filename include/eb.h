@@ -211,6 +211,22 @@ eb_status eb_step_host(eb_ctx* ctx, void* stream, const eb_batch* batch, uint32_
                        eb_policy policy, const eb_step_buffers* buf,
                        const float* h_logits, const void* h_x, void* h_out, eb_sched_result* h_res);
 
+/* Pipelined form of eb_step_host for independent steps: eb_step_host_submit enqueues the input copies
+ * on a copy stream of the context, the step on `stream` (after the copies) and the output copies on a
+ * second copy stream (after the step), and returns without waiting; eb_step_host_wait(slot) blocks until
+ * the outputs of the submission made with that slot are in host memory.  With two or more slots in use
+ * the copies of one step overlap the kernels of another; the kernels themselves still run one step
+ * after the other on `stream` (they share the workspace).  Rules: slot in [0, EB_HOST_SLOTS); a slot is
+ * reused only after its wait; buf->logits, buf->x, buf->sched and buf->out must be distinct buffers per
+ * slot in flight (the other buffers of eb_step_buffers may be shared by all slots); host buffers must
+ * stay valid, and should be pinned, until the wait returns.  The paper has no counterpart: it keeps the
+ * hidden states on the device between layers. */
+enum { EB_HOST_SLOTS = 4 };
+eb_status eb_step_host_submit(eb_ctx* ctx, void* stream, const eb_batch* batch, uint32_t route_mask, int32_t m,
+                              eb_policy policy, const eb_step_buffers* buf, const float* h_logits,
+                              const void* h_x, void* h_out, eb_sched_result* h_res, int32_t slot);
+eb_status eb_step_host_wait(eb_ctx* ctx, int32_t slot);
+
 /* ---- allocation-free variant --------------------------------------------------------------- */
 
 /* Largest packed token count eb_permute_noalloc accepts (its scratch is a fixed array). */

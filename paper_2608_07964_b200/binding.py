@@ -18,6 +18,7 @@ from .build import LIB, build_library
 EB_MAX_MB = 16
 EB_MAX_D = 16
 EB_META_LEN = 32
+EB_HOST_SLOTS = 4
 
 POLICY_MAXUTIL, POLICY_CUMUTIL, POLICY_DIFFPEAK, POLICY_ALL = 0, 1, 2, 3
 
@@ -45,6 +46,7 @@ class EbStepBuffers(C.Structure):
 SYMBOLS = ["eb_create", "eb_destroy", "eb_bind_weights", "eb_workspace_bytes", "eb_set_workspace",
            "eb_rows_capacity", "eb_groups_capacity", "eb_route", "eb_schedule", "eb_permute",
            "eb_expert_ffn_grouped", "eb_expert_ffn_device", "eb_combine", "eb_step", "eb_step_host",
+           "eb_step_host_submit", "eb_step_host_wait",
            "eb_permute_noalloc", "eb_selftest_bounded_wait", "eb_check_permutation",
            "eb_device_status", "eb_num_kernels", "eb_kernel_name", "eb_set_timing", "eb_kernel_ms",
            "eb_launch_count", "eb_status_string", "eb_last_error"]
@@ -82,6 +84,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.eb_combine.argtypes = [vp, vp, C.POINTER(EbBatch), vp, vp, vp, vp, vp]
     lib.eb_step.argtypes = [vp, vp, C.POINTER(EbBatch), u32, i32, i32, C.POINTER(EbStepBuffers)]
     lib.eb_step_host.argtypes = [vp, vp, C.POINTER(EbBatch), u32, i32, i32, C.POINTER(EbStepBuffers), vp, vp, vp, vp]
+    lib.eb_step_host_submit.argtypes = [vp, vp, C.POINTER(EbBatch), u32, i32, i32, C.POINTER(EbStepBuffers), vp, vp, vp, vp, i32]
+    lib.eb_step_host_wait.argtypes = [vp, i32]
     lib.eb_permute_noalloc.argtypes = [C.POINTER(EbConfig), vp, C.POINTER(EbBatch), vp, vp, vp, vp, vp, vp, vp, vp, vp,
                                        C.c_char_p, C.c_size_t]
     lib.eb_check_permutation.argtypes = [vp, vp, C.POINTER(EbBatch), vp, vp, vp, vp, vp, vp, vp, C.POINTER(i32)]
@@ -260,6 +264,40 @@ class MoEStep:
         self._check(self.lib.eb_step_host(self.ctx, _stream(), C.byref(batch.c), rm, m, policy, C.byref(self.bufs),
                                           h_logits.data_ptr(), h_x.data_ptr(), h_out.data_ptr(), C.addressof(h)))
         return _sched_dict(h, self.D)
+
+    def _slot_buffers(self, slot: int):
+        """Per-slot buffers of the pipelined host path: (eb_step_buffers, pinned host result, device tensors).
+        Inputs, schedule result and output are per slot; everything else is shared (the kernels of different
+        slots run one after the other)."""
+        if not hasattr(self, "_slots"):
+            self._slots = {}
+        if slot not in self._slots:
+            f32, bf = torch.float32, torch.bfloat16
+            mk = lambda shape, dt: torch.empty(shape, dtype=dt, device=self.dev)
+            logits, x = mk((self.max_tokens, self.E), f32), mk((self.max_tokens, self.H), bf)
+            sched = torch.zeros(C.sizeof(EbSchedResult), dtype=torch.uint8, device=self.dev)
+            out = mk((self.max_tokens, self.H), bf)
+            bufs = EbStepBuffers(*[t.data_ptr() for t in (
+                logits, x, self.topk_idx, self.topk_w, self.mb_load, self.mb_cnt, sched, self.group_off,
+                self.group_w, self.row_src, self.pos, self.xp, self.yp, self.step_meta, out)])
+            h_res = torch.zeros(C.sizeof(EbSchedResult), dtype=torch.uint8).pin_memory()   # pinned: the copy back is asynchronous
+            self._slots[slot] = (bufs, h_res, (logits, x, sched, out))
+        return self._slots[slot]
+
+    def step_host_submit(self, slot: int, batch: Batch, m: int, h_logits: torch.Tensor, h_x: torch.Tensor,
+                         h_out: torch.Tensor, policy: int = POLICY_MAXUTIL, route_mask: Optional[int] = None):
+        """Enqueues one host-to-host step on `slot` and returns; `step_host_wait(slot)` completes it."""
+        rm = ((1 << batch.n_mb) - 1) if route_mask is None else route_mask
+        assert not h_logits.is_cuda and not h_x.is_cuda and not h_out.is_cuda
+        bufs, h_res, _ = self._slot_buffers(slot)
+        self._check(self.lib.eb_step_host_submit(self.ctx, _stream(), C.byref(batch.c), rm, m, policy, C.byref(bufs),
+                                                 h_logits.data_ptr(), h_x.data_ptr(), h_out.data_ptr(),
+                                                 h_res.data_ptr(), slot))
+
+    def step_host_wait(self, slot: int) -> Dict:
+        self._check(self.lib.eb_step_host_wait(self.ctx, slot))
+        h_res = self._slot_buffers(slot)[1]
+        return _sched_dict(EbSchedResult.from_address(h_res.data_ptr()), self.D)
 
     # -- results and status --------------------------------------------------------------------
     def sched_result(self) -> Dict:

@@ -173,6 +173,13 @@ extern "C" eb_status eb_destroy(eb_ctx* c) {
   if (c->d_sched_scratch) cudaFree(c->d_sched_scratch);
   for (int i = 0; i < 2 * EBK_COUNT; ++i)
     if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+  for (int i = 0; i < EB_HOST_SLOTS; ++i) {
+    if (c->ev_in[i]) cudaEventDestroy(c->ev_in[i]);
+    if (c->ev_step[i]) cudaEventDestroy(c->ev_step[i]);
+    if (c->ev_out[i]) cudaEventDestroy(c->ev_out[i]);
+  }
+  if (c->s_in) cudaStreamDestroy(c->s_in);
+  if (c->s_out) cudaStreamDestroy(c->s_out);
   delete c;
   return EB_OK;
 }
@@ -266,6 +273,57 @@ extern "C" eb_status eb_step_host(eb_ctx* c, void* stream, const eb_batch* batch
   if (T) EB_CUDA(c, cudaMemcpyAsync(h_out, b->out, T * c->cfg.H * sizeof(bf16), cudaMemcpyDeviceToHost, st));
   if (h_res) EB_CUDA(c, cudaMemcpyAsync(h_res, b->sched, sizeof(eb_sched_result), cudaMemcpyDeviceToHost, st));
   EB_CUDA(c, cudaStreamSynchronize(st));
+  return EB_OK;
+}
+
+static eb_status host_pipeline_init(eb_ctx* c) {
+  if (c->s_in) return EB_OK;
+  EB_CUDA(c, cudaStreamCreateWithFlags(&c->s_in, cudaStreamNonBlocking));
+  EB_CUDA(c, cudaStreamCreateWithFlags(&c->s_out, cudaStreamNonBlocking));
+  for (int i = 0; i < EB_HOST_SLOTS; ++i) {
+    EB_CUDA(c, cudaEventCreateWithFlags(&c->ev_in[i], cudaEventDisableTiming));
+    EB_CUDA(c, cudaEventCreateWithFlags(&c->ev_step[i], cudaEventDisableTiming));
+    EB_CUDA(c, cudaEventCreateWithFlags(&c->ev_out[i], cudaEventDisableTiming));
+  }
+  return EB_OK;
+}
+
+extern "C" eb_status eb_step_host_submit(eb_ctx* c, void* stream, const eb_batch* batch, uint32_t route_mask, int32_t m,
+                                         eb_policy policy, const eb_step_buffers* b, const float* h_logits,
+                                         const void* h_x, void* h_out, eb_sched_result* h_res, int32_t slot) {
+  if (!c) return EB_ERR_INVALID_ARG;
+  if (slot < 0 || slot >= EB_HOST_SLOTS) return ebi_fail(c, EB_ERR_INVALID_ARG, "slot out of range");
+  if (c->slot_busy[slot]) return ebi_fail(c, EB_ERR_INVALID_ARG, "slot still in flight: call eb_step_host_wait first");
+  if (!h_logits || !h_x || !h_out) return ebi_fail(c, EB_ERR_INVALID_ARG, "null host buffer");
+  eb_status s = check_buffers(c, b);
+  if (s != EB_OK) return s;
+  BatchParams bp;
+  if ((s = ebi_make_batch(c, batch, &bp)) != EB_OK) return s;
+  if ((s = host_pipeline_init(c)) != EB_OK) return s;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t T = (size_t)bp.n_tok;
+  if (T) {
+    EB_CUDA(c, cudaMemcpyAsync(b->logits, h_logits, T * c->cfg.E * sizeof(float), cudaMemcpyHostToDevice, c->s_in));
+    EB_CUDA(c, cudaMemcpyAsync(b->x, h_x, T * c->cfg.H * sizeof(bf16), cudaMemcpyHostToDevice, c->s_in));
+  }
+  EB_CUDA(c, cudaEventRecord(c->ev_in[slot], c->s_in));
+  EB_CUDA(c, cudaStreamWaitEvent(st, c->ev_in[slot], 0));
+  if ((s = eb_step(c, stream, batch, route_mask, m, policy, b)) != EB_OK) return s;
+  EB_CUDA(c, cudaEventRecord(c->ev_step[slot], st));
+  EB_CUDA(c, cudaStreamWaitEvent(c->s_out, c->ev_step[slot], 0));
+  if (T) EB_CUDA(c, cudaMemcpyAsync(h_out, b->out, T * c->cfg.H * sizeof(bf16), cudaMemcpyDeviceToHost, c->s_out));
+  if (h_res) EB_CUDA(c, cudaMemcpyAsync(h_res, b->sched, sizeof(eb_sched_result), cudaMemcpyDeviceToHost, c->s_out));
+  EB_CUDA(c, cudaEventRecord(c->ev_out[slot], c->s_out));
+  c->slot_busy[slot] = true;
+  return EB_OK;
+}
+
+extern "C" eb_status eb_step_host_wait(eb_ctx* c, int32_t slot) {
+  if (!c) return EB_ERR_INVALID_ARG;
+  if (slot < 0 || slot >= EB_HOST_SLOTS) return ebi_fail(c, EB_ERR_INVALID_ARG, "slot out of range");
+  if (!c->slot_busy[slot]) return EB_OK;
+  c->slot_busy[slot] = false;
+  EB_CUDA(c, cudaEventSynchronize(c->ev_out[slot]));
   return EB_OK;
 }
 

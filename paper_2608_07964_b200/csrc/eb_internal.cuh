@@ -93,6 +93,10 @@ struct eb_ctx {
   int32_t max_chunks = 0, max_mtiles = 0, max_work1 = 0, max_work2 = 0, max_work1p = 0, max_work2p = 0;
 
   bool fused_attr_set = false;
+  // eb_step_host_submit / eb_step_host_wait: copy streams and per-slot events, created on first use
+  cudaStream_t s_in = nullptr, s_out = nullptr;
+  cudaEvent_t ev_in[EB_HOST_SLOTS] = {}, ev_step[EB_HOST_SLOTS] = {}, ev_out[EB_HOST_SLOTS] = {};
+  bool slot_busy[EB_HOST_SLOTS] = {};
   bool timing = false;
   cudaEvent_t ev[2 * EBK_COUNT] = {};
   bool ev_valid[EBK_COUNT] = {};

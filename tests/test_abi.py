@@ -29,6 +29,9 @@ def test_struct_layouts_match_the_header():
     assert binding.EbSchedResult.util_num.offset == 80
     assert ctypes.sizeof(binding.EbStepBuffers) == 15 * 8
     assert ctypes.sizeof(binding.EbConfig) == 48
+    text = open(os.path.join(ROOT, "include", "eb.h")).read()
+    for name in ("EB_MAX_MB", "EB_MAX_D", "EB_META_LEN", "EB_HOST_SLOTS"):
+        assert int(re.search(name + r"\s*=\s*(\d+)", text).group(1)) == getattr(binding, name), name
 
 
 def test_host_side_argument_errors_need_no_gpu():

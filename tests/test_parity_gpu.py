@@ -288,6 +288,49 @@ def test_step_and_step_host_match_the_five_calls():
     assert torch.equal(step.out[:T].cpu(), flipped)
 
 
+def test_pipelined_host_steps_match_the_blocking_call():
+    """Several host-to-host steps in flight on different slots, each with its own inputs: every slot's
+    result equals what the blocking call gives for the same inputs; slot misuse is refused."""
+    B = _binding()
+    wl = synth.workload("c1")
+    case = Hn.make_case(wl)
+    store = Hn.WeightStore(wl)
+    step, ref = _full_step(case, store, wl.m)
+    T = case.T_tot
+    batch = B.Batch(case.tok_off, case.layers)
+    n_slots = 4
+    xs = [case.x.clone() if s == 0 else torch.roll(case.x, shifts=s, dims=0) for s in range(n_slots)]
+    h_logits = case.logits.clone().pin_memory()
+    h_xs = [x.clone().pin_memory() for x in xs]
+    want = []
+    for s in range(n_slots):
+        h_out = torch.full((T, wl.H), -7.0, dtype=torch.bfloat16).pin_memory()
+        step.eb_step_host(batch, wl.m, h_logits, h_xs[s], h_out)
+        want.append(h_out.clone())
+    run0 = [j for j in range(len(case.tok_off) - 1) if (ref["sched"]["run_mask"] >> j) & 1][0]
+    a0, b0 = case.tok_off[run0], case.tok_off[run0 + 1]
+    assert not torch.equal(want[0][a0:b0], want[1][a0:b0])
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for rounds in range(3):
+            h_outs = [torch.full((T, wl.H), -7.0, dtype=torch.bfloat16).pin_memory() for _ in range(n_slots)]
+            for s in range(n_slots):
+                step.step_host_submit(s, batch, wl.m, h_logits, h_xs[s], h_outs[s])
+            with pytest.raises(B.EbError):
+                step.step_host_submit(1, batch, wl.m, h_logits, h_xs[1], h_outs[1])   # slot 1 is still in flight
+            for s in reversed(range(n_slots)):
+                res = step.step_host_wait(s)
+                assert res["run_mask"] == ref["sched"]["run_mask"]
+                for j in range(len(case.tok_off) - 1):      # rows of deferred micro-batches are not written
+                    if (res["run_mask"] >> j) & 1:
+                        a, b = case.tok_off[j], case.tok_off[j + 1]
+                        assert torch.equal(h_outs[s][a:b], want[s][a:b]), (rounds, s, j)
+        assert step.step_host_wait(2)["run_mask"] == ref["sched"]["run_mask"]   # waiting on an idle slot is a no-op
+        with pytest.raises(B.EbError):
+            step.step_host_submit(B.EB_HOST_SLOTS, batch, wl.m, h_logits, h_xs[0], h_outs[0])
+    assert step.device_status() == 0
+
+
 def test_deferred_micro_batch_keeps_its_routing():
     B = _binding()
     wl = synth.workload("c1")
