@@ -287,7 +287,7 @@ rank_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ 
 
 // ---- fused kernel for small steps --------------------------------------------------------------
 // hist + sizes + scan + rank in one block when the step has at most kFusedMaxChunks chunks and
-// kFusedMaxGroups group slots: the per-chunk tables live in shared memory and three kernel boundaries
+// kFusedMaxGroups group slots: the routing decisions and the per-chunk tables live in shared memory and three kernel boundaries
 // disappear (these kernels are pure latency on small steps).  Same arithmetic, same results.
 constexpr int kFusedMaxChunks = 32;
 constexpr int kFusedMaxGroups = 4096;
@@ -304,13 +304,28 @@ permute_fused_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __re
   __shared__ int s_warp[32];
   __shared__ int s_carry;
   const int E = mp.E, K = mp.K, S = mp.S, KS = K + S, D = mp.D;
-  int* s_tab = s_dyn;                          // [n_chunks][E]: histogram, then first rank of the chunk in its group
-  int* s_goff = s_dyn + bp.n_chunks * E;       // [G + 1]: group sizes, then offsets
+  __shared__ int s_e2d[EB_MAX_E], s_e_local[EB_MAX_E], s_dev_list[EB_MAX_E];
+  int* s_topk = s_dyn;                         // [n_tok][K]: the routing decisions
+  int* s_tab = s_topk + bp.n_tok * K;          // [n_chunks][E]: histogram, then first rank of the chunk in its group
+  int* s_goff = s_tab + bp.n_chunks * E;       // [G + 1]: group sizes, then offsets
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // every global read of the kernel is issued here, together: the phases below are chains of block barriers
+  // and would otherwise each pay a trip to memory
   const uint32_t run = res->run_mask;
+  for (int i = tid; i < bp.n_tok * K; i += kFusedThreads) s_topk[i] = topk_idx[i];
+  for (int e = tid; e < E; e += kFusedThreads) {
+    s_e2d[e] = mp.e2d[e];
+    s_e_local[e] = mp.e_local[e];
+    s_dev_list[e] = mp.dev_list[e];
+  }
   __shared__ StepShape ss;
+  __shared__ int s_home[EB_MAX_MB][EB_MAX_D + 1];   // first local token of every home device, per micro-batch
   if (tid == 0) s_carry = 0;
   if (tid <= D) s_dev_off[tid] = mp.dev_off[tid];
+  if (tid < EB_MAX_MB * (EB_MAX_D + 1)) {
+    const int j = tid / (EB_MAX_D + 1), d = tid % (EB_MAX_D + 1);
+    if (j < bp.n_mb && d <= D) s_home[j][d] = home_start(d, bp.tok_off[j + 1] - bp.tok_off[j], D);
+  }
   step_shape_block(bp, run, &ss);
   const int G = ss.nl * (E + D * S);
 
@@ -323,7 +338,7 @@ permute_fused_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __re
     if ((run >> j) & 1u) {
       const int t0 = bp.tok_off[j] + (c - bp.chunk_off[j]) * 32;
       const int nt = min(32, bp.tok_off[j + 1] - t0);
-      for (int a = lane; a < nt * K; a += 32) atomicAdd(&h[topk_idx[(size_t)t0 * K + a]], 1);
+      for (int a = lane; a < nt * K; a += 32) atomicAdd(&h[s_topk[t0 * K + a]], 1);
     }
   }
   __syncthreads();
@@ -338,12 +353,9 @@ permute_fused_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __re
     int tot = 0;
     if (local >= n_d) {
       for (int j = 0; j < bp.n_mb; ++j)
-        if (ss.rank_of_mb[j] == lr) {
-          const int T = bp.tok_off[j + 1] - bp.tok_off[j];
-          tot += home_start(d + 1, T, D) - home_start(d, T, D);
-        }
+        if (ss.rank_of_mb[j] == lr) tot += s_home[j][d + 1] - s_home[j][d];
     } else {
-      const int e = mp.dev_list[s_dev_off[d] + local];
+      const int e = s_dev_list[s_dev_off[d] + local];
       for (int j = 0; j < bp.n_mb; ++j) {
         if (ss.rank_of_mb[j] != lr) continue;
         for (int c = bp.chunk_off[j]; c < bp.chunk_off[j + 1]; ++c) {
@@ -388,7 +400,7 @@ permute_fused_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __re
       const int n_d = s_dev_off[d + 1] - s_dev_off[d];
       const int rel = g - ss.nl * (s_dev_off[d] + d * S);
       const int lr = rel / (n_d + S), local = rel % (n_d + S);
-      const int slot = local < n_d ? mp.dev_list[s_dev_off[d] + local] : E + (local - n_d);
+      const int slot = local < n_d ? s_dev_list[s_dev_off[d] + local] : E + (local - n_d);
       group_w[g] = ss.act_layer[lr] * (E + S) + slot;
     }
     __syncthreads();
@@ -420,12 +432,12 @@ permute_fused_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __re
     const int lr = ss.rank_of_mb[j];
     int* next = s_tab + c * E;
     for (int e = lane; e < E; e += 32)
-      next[e] += s_goff[group_id(s_dev_off, S, ss.nl, mp.e2d[e], lr, mp.e_local[e])];
+      next[e] += s_goff[group_id(s_dev_off, S, ss.nl, s_e2d[e], lr, s_e_local[e])];
     __syncwarp();
     for (int a0 = 0; a0 < nt * K; a0 += 32) {
       const int a = a0 + lane;
       const bool valid = a < nt * K;
-      const int e = valid ? topk_idx[(size_t)t0 * K + a] : -1 - lane;
+      const int e = valid ? s_topk[t0 * K + a] : -1 - lane;
       const unsigned peers = __match_any_sync(0xffffffffu, e);
       const int before = __popc(peers & ((1u << lane) - 1u));
       if (valid) {
@@ -439,18 +451,15 @@ permute_fused_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __re
       __syncwarp();
     }
     if (S > 0 && lane < nt) {
-      const int T = bp.tok_off[j + 1] - bp.tok_off[j];
       const int tl = t0 + lane - bp.tok_off[j];
-      const int d = home_device(tl, T, D);
+      int d = 0;   // home device: the last one whose first token is not beyond tl
+      while (d + 1 < D && tl >= s_home[j][d + 1]) ++d;
       int before = 0;
       for (int j2 = 0; j2 < j; ++j2)
-        if (ss.rank_of_mb[j2] == lr) {
-          const int T2 = bp.tok_off[j2 + 1] - bp.tok_off[j2];
-          before += home_start(d + 1, T2, D) - home_start(d, T2, D);
-        }
+        if (ss.rank_of_mb[j2] == lr) before += s_home[j2][d + 1] - s_home[j2][d];
       const int n_d = s_dev_off[d + 1] - s_dev_off[d];
       for (int s2 = 0; s2 < S; ++s2) {
-        const int p = s_goff[group_id(s_dev_off, S, ss.nl, d, lr, n_d + s2)] + before + (tl - home_start(d, T, D));
+        const int p = s_goff[group_id(s_dev_off, S, ss.nl, d, lr, n_d + s2)] + before + (tl - s_home[j][d]);
         pos[(size_t)(t0 + lane) * KS + K + s2] = p;
         row_src[p] = t0 + lane;
       }
@@ -518,13 +527,13 @@ extern "C" eb_status eb_permute(eb_ctx* c, void* stream, const eb_batch* batch, 
   const int chunk_blocks = (bp.n_chunks + kWarps - 1) / kWarps;
   if (bp.n_chunks <= kFusedMaxChunks && gcap <= kFusedMaxGroups) {
     // small step: one block does histogram, sizes, scan and ranks
-    const size_t smem = sizeof(int) * ((size_t)kFusedMaxChunks * EB_MAX_E + kFusedMaxGroups + 1);
+    const size_t smem = sizeof(int) * ((size_t)kFusedMaxChunks * EB_MAX_E + kFusedMaxGroups + 1 + (size_t)kFusedMaxChunks * 32 * EB_MAX_K);
     if (!c->fused_attr_set) {   // per context: function attributes belong to the current device
       EB_CUDA(c, cudaFuncSetAttribute(permute_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
       c->fused_attr_set = true;
     }
     KernelTimer timer(c, EBK_PERMUTE_FUSED, st);
-    ebi_launch(permute_fused_kernel, dim3(1), dim3(kFusedThreads), sizeof(int) * ((size_t)bp.n_chunks * c->cfg.E + gcap + 1),
+    ebi_launch(permute_fused_kernel, dim3(1), dim3(kFusedThreads), sizeof(int) * ((size_t)bp.n_chunks * c->cfg.E + gcap + 1 + (size_t)bp.n_tok * c->cfg.K),
                st, c->mp, bp, d_res, topk_idx, group_off, group_w, pos, row_src, step_meta);
   } else {
     if (bp.n_chunks > 0) {

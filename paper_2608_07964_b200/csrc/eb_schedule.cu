@@ -52,6 +52,20 @@ __device__ __forceinline__ Cand make_cand(const long long* w, int D, int n, unsi
   return c;
 }
 
+// best candidate of the warp, in every lane
+__device__ __forceinline__ Cand warp_best(Cand c) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    Cand oth;
+    oth.num = __shfl_xor_sync(0xffffffffu, c.num, o);
+    oth.peak = __shfl_xor_sync(0xffffffffu, c.peak, o);
+    oth.n = __shfl_xor_sync(0xffffffffu, c.n, o);
+    oth.sub = __shfl_xor_sync(0xffffffffu, c.sub, o);
+    if (better(oth, c)) c = oth;
+  }
+  return c;
+}
+
 __global__ void __launch_bounds__(kThreads)
 schedule_kernel(int D, int n_mb, uint32_t pool_mask, int m, int policy, const int32_t* __restrict__ mb_load,
                 eb_sched_result* __restrict__ res, Cand* __restrict__ block_best, unsigned* __restrict__ block_counter) {
@@ -73,11 +87,7 @@ schedule_kernel(int D, int n_mb, uint32_t pool_mask, int m, int policy, const in
     s_load[j][d] = (j < n_mb && d < D) ? mb_load[j * D + d] : 0;
   }
   const int np = __popc(pool_mask);
-  if (tid == 0) {
-    int k = 0;
-    for (int j = 0; j < EB_MAX_MB; ++j)
-      if ((pool_mask >> j) & 1u) s_member[k++] = j;
-  }
+  if (tid < EB_MAX_MB && ((pool_mask >> tid) & 1u)) s_member[__popc(pool_mask & ((1u << tid) - 1u))] = tid;
   __syncthreads();
 
   if (np <= m || policy == EB_POLICY_ALL) {
@@ -111,25 +121,18 @@ schedule_kernel(int D, int n_mb, uint32_t pool_mask, int m, int policy, const in
       Cand c = make_cand(w, D, n, sub);
       if (better(c, best)) best = c;
     }
-    // warp then block reduction under the total order
-    for (int o = 16; o > 0; o >>= 1) {
-      Cand oth;
-      oth.num = __shfl_xor_sync(0xffffffffu, best.num, o);
-      oth.peak = __shfl_xor_sync(0xffffffffu, best.peak, o);
-      oth.n = __shfl_xor_sync(0xffffffffu, best.n, o);
-      oth.sub = __shfl_xor_sync(0xffffffffu, best.sub, o);
-      if (better(oth, best)) best = oth;
-    }
+    // warp then block reduction under the total order (any reduction order gives the same winner)
+    best = warp_best(best);
     if ((tid & 31) == 0) s_best[tid >> 5] = best;
     __syncthreads();
+    if (tid < 32) {
+      Cand b = warp_best(s_best[tid]);
+      if (tid == 0) s_best[0] = b;
+    }
     if (gridDim.x > 1) {
       // every block leaves its best candidate in global memory; the block that arrives last reduces them
-      // (the total order makes the result independent of which block that is)
       if (tid == 0) {
-        Cand b = s_best[0];
-        for (int i = 1; i < kThreads / 32; ++i)
-          if (better(s_best[i], b)) b = s_best[i];
-        block_best[blockIdx.x] = b;
+        block_best[blockIdx.x] = s_best[0];
         __threadfence();
         const unsigned arrived = atomicAdd(block_counter, 1u);
         s_last = arrived == gridDim.x - 1;
@@ -144,25 +147,15 @@ schedule_kernel(int D, int n_mb, uint32_t pool_mask, int m, int policy, const in
           const Cand o = block_best[i];
           if (better(o, b)) b = o;
         }
-        for (int o = 16; o > 0; o >>= 1) {
-          Cand oth;
-          oth.num = __shfl_xor_sync(0xffffffffu, b.num, o);
-          oth.peak = __shfl_xor_sync(0xffffffffu, b.peak, o);
-          oth.n = __shfl_xor_sync(0xffffffffu, b.n, o);
-          oth.sub = __shfl_xor_sync(0xffffffffu, b.sub, o);
-          if (better(oth, b)) b = oth;
-        }
+        b = warp_best(b);
         if (tid == 0) {
           s_best[0] = b;
           *block_counter = 0;   // ready for the next call
         }
       }
-      __syncthreads();
     }
     if (tid == 0) {
-      Cand b = s_best[0];
-      for (int i = 1; gridDim.x == 1 && i < kThreads / 32; ++i)
-        if (better(s_best[i], b)) b = s_best[i];
+      const Cand b = s_best[0];
       uint32_t mask = 0;
       for (int k = 0; k < np; ++k)
         if ((b.sub >> k) & 1u) mask |= 1u << s_member[k];
@@ -241,23 +234,30 @@ schedule_kernel(int D, int n_mb, uint32_t pool_mask, int m, int policy, const in
     }
   }
   __syncthreads();
-  if (tid == 0) {
-    uint32_t run = s_run;
-    long long num = 0, peak = 0;
-    for (int d = 0; d < EB_MAX_D; ++d) {
-      long long v = 0;
+  if (tid < 32) {
+    // lane d sums the chosen micro-batches' load on device d (zero beyond D); the warp adds and maximises
+    const uint32_t run = s_run;
+    long long v = 0;
+    if (tid < EB_MAX_D) {
       for (int j = 0; j < EB_MAX_MB; ++j)
-        if ((run >> j) & 1u) v += s_load[j][d];
-      res->joint_load[d] = (int32_t)v;
-      num += v;
-      peak = v > peak ? v : peak;
+        if ((run >> j) & 1u) v += s_load[j][tid];
+      res->joint_load[tid] = (int32_t)v;
     }
-    res->run_mask = run;
-    res->defer_mask = pool_mask & ~run;
-    res->n_run = __popc(run);
-    res->status = EB_OK;
-    res->util_num = num;
-    res->util_den = (long long)D * peak;
+    long long num = v, peak = v;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      num += __shfl_xor_sync(0xffffffffu, num, o);
+      const long long p2 = __shfl_xor_sync(0xffffffffu, peak, o);
+      peak = p2 > peak ? p2 : peak;
+    }
+    if (tid == 0) {
+      res->run_mask = run;
+      res->defer_mask = pool_mask & ~run;
+      res->n_run = __popc(run);
+      res->status = EB_OK;
+      res->util_num = num;
+      res->util_den = (long long)D * peak;
+    }
   }
 }
 
