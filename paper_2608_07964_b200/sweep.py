@@ -1,6 +1,6 @@
 """Skew / micro-batch sweep on the 64-expert, top-6, hidden-2048 shape (8 layers, 8 virtual devices).
 
-    python -m paper_2608_07964_b200.sweep [--out results.md] [--policy 0]
+    python -m paper_2608_07964_b200.sweep [--out results.md] [--policy 0] [--ep | --msweep | --latency | --sched]
 
 For every point (Zipf s, micro-batch count N, tokens per micro-batch T) it reports
   * whole-run under-utilisation 1 - u of Algorithm 1 driven on the GPU (route + schedule every
@@ -121,6 +121,36 @@ def schedule_latency_report(args, dev):
     return lines
 
 
+def m_sweep(args, dev, weights):
+    """Minimum combination size sweep (the paper's micro-batching ablation): for every micro-batch count N and
+    every m from 1 to N, whole-run under-utilisation of Algorithm 1 under the three policies, the number of steps,
+    and the ratio of effective to maximum workload summed over steps (max_d sum_j w_j against sum_j max_d w_j,
+    the two curves of the paper's per-step plot)."""
+    lines = ["| s | N | m | steps (MaxUtil) | idle MaxUtil | idle CumUtil | idle DiffPeak | idle alone | effective / maximum workload (MaxUtil) |",
+             "|---|---|---|---|---|---|---|---|---|"]
+    for s in (0.5, 1.0):
+        for N in (2, 4, 8, 16):
+            wl = synth.workload_c5(N, 128, s)
+            bias = synth.zipf_bias(wl)
+            step = B.from_workload(wl, device=dev)
+            step.bind_weights(*weights)
+            logits_of = lambda j, l: synth.logits_for(wl, j, l, dev, bias)
+            for m in range(1, N + 1):
+                res = {}
+                for name, pol in (("max", B.POLICY_MAXUTIL), ("cum", B.POLICY_CUMUTIL), ("diff", B.POLICY_DIFFPEAK)):
+                    tr = driver.run_load_trace(step, wl.tok_off, wl.L, m, pol, logits_of)
+                    res[name] = (driver.idle_fractions(tr, wl.D), tr)
+                tr = res["max"][1]
+                eff = sum(max(st["joint_load"][:wl.D]) for st in tr)
+                mx = sum(max(w) for st in tr for w in st["member_loads"].values())
+                f = res["max"][0]
+                lines.append(f"| {s} | {N} | {m} | {f['steps']} | {f['idle_cross_layer']:.3f} | {res['cum'][0]['idle_cross_layer']:.3f} | "
+                             f"{res['diff'][0]['idle_cross_layer']:.3f} | {f['idle_each_alone']:.3f} | {eff / mx:.3f} |")
+                print(lines[-1], flush=True)
+            step.close()
+    return lines
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--out", default=None)
@@ -129,6 +159,7 @@ def main(argv=None):
     ap.add_argument("--ep", action="store_true", help="expert-parallel size sweep instead of the skew sweep")
     ap.add_argument("--latency", action="store_true", help="emulated expert-parallel latency of whole runs")
     ap.add_argument("--sched", action="store_true", help="time of one scheduling call per policy")
+    ap.add_argument("--msweep", action="store_true", help="minimum combination size sweep")
     args = ap.parse_args(argv)
     dev = "cuda:0"
     if args.sched:
@@ -145,6 +176,12 @@ def main(argv=None):
         return 0
     base = synth.workload_c5(2, 16, 0.0)
     weights = tuple(synth.all_weights(base, k, dev) for k in ("gate", "up", "down"))
+    if args.msweep:
+        text = "\n".join(m_sweep(args, dev, weights)) + "\n"
+        if args.out:
+            with open(args.out, "w") as f:
+                f.write(text)
+        return 0
     if args.ep:
         text = "\n".join(ep_size_sweep(args, dev, weights)) + "\n"
         if args.out:
