@@ -26,7 +26,8 @@
 // gate/up: CTA 0 the gate rows, CTA 1 the up rows), and the leader CTA issues tcgen05.mma
 // cta_group::2 (M = 256) that reads both halves.  A stage shrinks from 48 KB to 32 KB per CTA for the
 // same tensor-core time, so the ring deepens to 7 stages and L2 traffic per flop drops by a third -
-// that is what the tensor-bound regime needs.  No load is multicast; only tcgen05.commit is.
+// that is what the tensor-bound regime needs.  Every CTA fetches its own operands; only the tcgen05.commit
+// that frees a stage is delivered to both CTAs of the pair.
 //
 // Every wait on an mbarrier is bounded: on expiry the kernel records EB_ERR_TIMEOUT in the
 // context status word, lets copies in flight land, frees its TMEM and returns.
@@ -133,7 +134,8 @@ __device__ __forceinline__ void cluster_sync_all() {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
-// TMA loads whose completion is counted on a barrier that may live in the peer CTA (never multicast)
+// TMA loads whose completion is counted on a barrier that may live in the peer CTA (the data goes to the
+// issuing CTA only)
 __device__ __forceinline__ void tma_pair_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
