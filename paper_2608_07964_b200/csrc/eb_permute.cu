@@ -39,24 +39,31 @@ __device__ __forceinline__ int home_device(int tl, int T, int D) {
 // micro-batch, the result lands in shared memory.  Ends with a block barrier.
 __device__ __forceinline__ void step_shape_block(const BatchParams& bp, uint32_t run, StepShape* out) {
   const int j = threadIdx.x;
-  if (j < EB_MAX_MB) {
+  if (j < 32) {   // warp 0; lanes 0..15 each own one micro-batch
     const bool sel = j < bp.n_mb && ((run >> j) & 1u);
-    int below = 0, total = 0;
-    bool first_of_layer = sel;
-    for (int i = 0; i < bp.n_mb; ++i) {
-      if (!((run >> i) & 1u)) continue;
-      bool first = true;   // is i the first chosen micro-batch sitting at its layer?
-      for (int i2 = 0; i2 < i; ++i2)
-        if (((run >> i2) & 1u) && bp.layer[i2] == bp.layer[i]) first = false;
-      if (first) {
-        ++total;
-        if (sel && bp.layer[i] < bp.layer[j]) ++below;
-      }
-      if (sel && i < j && bp.layer[i] == bp.layer[j]) first_of_layer = false;
+    const int my_layer = j < bp.n_mb ? bp.layer[j] : -1;
+    // is j the first chosen micro-batch sitting at its layer?
+    bool first = sel;
+    for (int i = 0; i < EB_MAX_MB; ++i) {
+      const int li = __shfl_sync(0xffffffffu, my_layer, i);
+      const bool si = (run >> i) & 1u;
+      if (i < j && si && li == my_layer) first = false;
     }
-    out->rank_of_mb[j] = sel ? below : -1;
-    if (first_of_layer) out->act_layer[below] = bp.layer[j];
-    if (j == 0) out->nl = total;
+    // distinct chosen layers below mine, and in total
+    int below = 0, total = 0;
+    for (int i = 0; i < EB_MAX_MB; ++i) {
+      const int li = __shfl_sync(0xffffffffu, my_layer, i);
+      const bool fi = __shfl_sync(0xffffffffu, (int)first, i) != 0;
+      if (fi) {
+        ++total;
+        if (li < my_layer) ++below;
+      }
+    }
+    if (j < EB_MAX_MB) {
+      out->rank_of_mb[j] = sel ? below : -1;
+      if (first) out->act_layer[below] = my_layer;
+      if (j == 0) out->nl = total;
+    }
   }
   __syncthreads();
 }
