@@ -97,3 +97,26 @@ def test_full_chain_matches_oracle_chain_on_c1():
     assert n_steps == len(got["steps"])
     xg = got["x"].float().cpu().numpy()
     assert Hn.within_bar(xg, x), f"final hidden states off by {Hn.worst(xg, x):.2f} x bar"
+
+
+def test_emulated_latency_accounts_every_step_and_device():
+    """The emulated expert-parallel latency loop takes the same steps as the load trace, costs each step its
+    slowest virtual device, and with `alone` executes every (micro-batch, layer) workload by itself."""
+    from paper_2608_07964_b200 import binding as B, driver
+    wl = synth.workload("c1")
+    bias = synth.zipf_bias(wl)
+    store = Hn.WeightStore(wl)
+    step = B.from_workload(wl)
+    step.bind_weights(store.gate, store.up, store.down)
+    x0 = torch.cat([synth.hidden_for(wl, j, 0, "cuda") for j in range(wl.N)], 0)
+    logits_of = lambda j, l: synth.logits_for(wl, j, l, "cuda", bias)
+    trace = driver.run_load_trace(step, wl.tok_off, wl.L, wl.m, O.POLICY_MAXUTIL, logits_of)
+    r = driver.run_emulated_latency(step, wl.tok_off, wl.L, wl.D, wl.m, O.POLICY_MAXUTIL, logits_of, x0)
+    assert r["steps"] == len(trace)
+    assert r["latency_ms"] > 0 and 0 < r["busy_ms"] <= wl.D * r["latency_ms"] * (1 + 1e-6)
+    assert 0.0 <= r["idle_time"] < 1.0
+    alone = driver.run_emulated_latency(step, wl.tok_off, wl.L, wl.D, 1, O.POLICY_ALL, logits_of, x0, alone=True)
+    assert alone["steps"] == wl.N * wl.L
+    lock = driver.run_emulated_latency(step, wl.tok_off, wl.L, wl.D, wl.N, O.POLICY_ALL, logits_of, x0)
+    assert lock["steps"] == wl.L
+    assert step.device_status() == 0
