@@ -14,18 +14,22 @@ What each function follows:
 * ``group_table`` / ``permute`` - the dispatch of Section 2.2 written as a stable grouping of
                      (token, expert) assignments by (virtual device, layer, expert).
 * ``expert_ffn``   - ``expert_i(.)`` of Eq. 1 as a bias-free SwiGLU MLP.
-* ``combine``      - Eq. 1, the weighted aggregation.
+* ``combine``      - Eq. 1, the weighted aggregation; optionally h_{l+1} = h'_l + MLP(h'_l) of Section 2.1.
 * ``dense_masked_moe`` - Eq. 1 evaluated with every expert on every token and a 0/weight mask:
                      a brute-force cross-check that uses no permutation at all.
 * ``run_algorithm1`` - Algorithm 1 on load vectors (which workloads run at which step).
+* ``same_peak_windows`` - the count of N-consecutive layers with the same skew device (the paper's
+                     table of worst-case occurrences, Section 4.1).
 * ``idle_*``       - under-utilisation ``1 - u`` (Section 5, Metrics) for the cross-layer run,
                      for each workload executed alone, and for lock-step execution.
 
-Readings taken where the paper is silent are listed in the repository's design notes; the ones
-with no independent pin ("parity unpinned") are: the placement of shared experts (replicated on
-every virtual device, serving that device's home tokens, not counted in scheduling loads), the
-MaxUtil tie rule (higher U, then larger set, then smaller bitmask), and how CumUtil / DiffPeak
-are topped up to ``m`` members.
+Readings taken where the paper is silent are listed in the repository's design notes.  Three of
+them are choices the paper cannot confirm ("parity unpinned" in that sense): the placement of
+shared experts (replicated on every virtual device, serving that device's home tokens, not
+counted in scheduling loads), the MaxUtil tie rule (higher U, then larger set, then smaller
+bitmask), and how CumUtil / DiffPeak are topped up to ``m`` members (best utilisation of the
+union, ties to the lower index).  What each reading *is* is fixed by hand-worked examples in the
+test-suite, so a slip in their code fails a test; that the paper means them is not checkable.
 
 Floating point is fp32 by default (the precision the parity bar is stated in); every float
 function takes ``dtype`` so the tests can repeat it in fp64 to bound the oracle's own error.
@@ -284,9 +288,12 @@ def expert_ffn(xp: np.ndarray, group_off: np.ndarray, group_w: np.ndarray,
     return y
 
 
-def combine(y: np.ndarray, pos: np.ndarray, topk_w: np.ndarray, K: int, S: int, dtype=np.float32) -> np.ndarray:
+def combine(y: np.ndarray, pos: np.ndarray, topk_w: np.ndarray, K: int, S: int, dtype=np.float32,
+            residual: np.ndarray = None) -> np.ndarray:
     """Eq. 1: out[t] = sum_k W[t,k] * y[pos[t,k]] + sum_s y[pos[t,K+s]] (k ascending, then s).
 
+    With `residual` (the MoE block's input h'_l, one row per token) the result is the next hidden
+    state of Section 2.1, h_{l+1} = h'_l + MLP(h'_l): the row of `residual` is added last.
     Rows of tokens with pos < 0 (micro-batch not selected) are returned as zeros and flagged in
     the boolean vector that comes with the result.
     """
@@ -302,7 +309,10 @@ def combine(y: np.ndarray, pos: np.ndarray, topk_w: np.ndarray, K: int, S: int, 
             acc = acc + dtype(topk_w[t, k]) * y[pos[t, k]].astype(dtype)
         for s in range(S):
             acc = acc + y[pos[t, K + s]].astype(dtype)
-        out[t] = acc
+        if residual is not None:
+            out[t] = acc + residual[t].astype(dtype)
+        else:
+            out[t] = acc
         done[t] = True
     return out, done
 
@@ -362,6 +372,21 @@ def run_algorithm1(load_of: Callable[[int, int], Sequence[int]], N: int, L: int,
             if l[j] >= L:
                 pool &= ~(1 << j)
     return steps
+
+
+def same_peak_windows(loads_by_layer: Sequence[Sequence[int]], n: int) -> Tuple[int, int]:
+    """How many windows of n consecutive layers have their workload skewed to the same device
+    (the statistic of the paper's table on consecutive layers: the worst case of Section 4.1,
+    where combining gains nothing).  `loads_by_layer[l]` is the load vector of layer l; the skew
+    device is the peak device, lowest index among equal maxima.  Returns (count, windows) with
+    windows = L - n + 1."""
+    peaks = [_peak_device(w) for w in loads_by_layer]
+    windows = max(len(peaks) - n + 1, 0)
+    count = 0
+    for l in range(windows):
+        if all(peaks[l + i] == peaks[l] for i in range(1, n)):
+            count += 1
+    return count, windows
 
 
 def idle_cross_layer(steps: List[Dict], D: int) -> Tuple[int, int]:

@@ -246,6 +246,32 @@ def test_uniform_routing_gives_zero_idle_and_full_run_set():
     assert len(steps) == 3 and O.idle_cross_layer(steps, D)[0] == 0
 
 
+def test_combine_with_residual_by_hand():
+    # two expert rows, one token with weights 1/4 and 3/4: 0.25*(4, 8) + 0.75*(8, -4) = (7, -1); plus h' = (1, 10)
+    y = np.array([[4.0, 8.0], [8.0, -4.0]])
+    pos = np.array([[0, 1], [-1, -1]], dtype=np.int32)
+    w = np.array([[0.25, 0.75], [0.5, 0.5]])
+    h = np.array([[1.0, 10.0], [5.0, 5.0]])
+    out, done = O.combine(y, pos, w, 2, 0, dtype=np.float64)
+    assert out.tolist() == [[7.0, -1.0], [0.0, 0.0]] and done.tolist() == [True, False]
+    nxt, done = O.combine(y, pos, w, 2, 0, dtype=np.float64, residual=h)
+    assert nxt.tolist() == [[8.0, 9.0], [0.0, 0.0]] and done.tolist() == [True, False]
+
+
+def test_same_peak_windows_by_hand():
+    # peaks 0, 0, 1, 0 (tied maxima -> lower device), 0: pairs (0,0) (0,1) (1,0) (0,0) -> 2 of 4; no triple of 3
+    loads = [(3, 1), (2, 0), (0, 5), (1, 1), (4, 2)]
+    assert O.same_peak_windows(loads, 2) == (2, 4)
+    assert O.same_peak_windows(loads, 3) == (0, 3)
+    # peaks 1, 1, 1, 0: pairs -> 2 of 3, triples -> 1 of 2; a window longer than the sequence -> 0 of 0
+    loads = [(0, 2), (1, 9), (3, 4), (5, 0)]
+    assert O.same_peak_windows(loads, 2) == (2, 3)
+    assert O.same_peak_windows(loads, 3) == (1, 2)
+    assert O.same_peak_windows(loads, 5) == (0, 0)
+    # 48 layers give 47 pairs and 46 triples, the denominators the paper's table prints
+    assert O.same_peak_windows([(1, 0)] * 48, 2) == (47, 47) and O.same_peak_windows([(1, 0)] * 48, 3) == (46, 46)
+
+
 # ------------------------------------------------------------------ routing
 def test_route_full_k_is_softmax_and_k1_is_argmax():
     from scipy.special import softmax
@@ -372,6 +398,11 @@ def test_pipeline_equals_dense_masked_bruteforce():
         ref = O.dense_masked_moe(x, idx, w, tok_layer, E, S, get, dtype=np.float64)
         assert (done == (tok_layer >= 0)).all()
         assert np.allclose(out, ref, rtol=1e-11, atol=1e-11)
+        # Section 2.1: h_{l+1} = h' + MLP(h'); the brute-force MoE output plus the input, no shared code path
+        nxt, _ = O.combine(y, pos, w, K, S, dtype=np.float64, residual=x)
+        sel = tok_layer >= 0
+        assert np.allclose(nxt[sel], (ref + x.astype(np.float64))[sel], rtol=1e-11, atol=1e-11)
+        assert (nxt[~sel] == 0).all()
         # fp32 oracle against the fp64 one: bounds the oracle's own rounding error
         y32 = O.expert_ffn(xp, goff, gw, get, dtype=np.float32)
         out32, _ = O.combine(y32, pos, w, K, S, dtype=np.float32)
