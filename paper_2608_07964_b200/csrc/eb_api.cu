@@ -82,14 +82,15 @@ static size_t carve(eb_ctx* c, char* base) {
   c->max_work1 = c->max_mtiles * ((g.I + 127) / 128);
   c->max_work2 = c->max_mtiles * ((g.H + 255) / 256);
   const int max_ptiles = rows / 256 + gcap;
-  c->max_work1p = max_ptiles * ((g.I + 127) / 128);
-  c->max_work2p = max_ptiles * ((g.H + 255) / 256);
+  c->max_work1p = max_ptiles * ((g.I + 255) / 256);   // pair tiles: 256 outputs (gate/up), 512 outputs (down)
+  c->max_work2p = max_ptiles * ((g.H + 511) / 512);
   c->chunk_hist = (int32_t*)take(sizeof(int32_t) * (size_t)c->max_chunks * g.E);
   c->chunk_base = (int32_t*)take(sizeof(int32_t) * (size_t)c->max_chunks * g.E);
   c->group_size = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
   c->mtile_pref = (int32_t*)take(sizeof(int32_t) * (size_t)(gcap + 1));
   c->ptile_pref = (int32_t*)take(sizeof(int32_t) * (size_t)(gcap + 1));
   c->pgroup = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
+  c->ppgroup = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
   c->pchunks = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
   c->work_count = (int32_t*)take(sizeof(int32_t) * 16);
   c->work1 = (int4*)take(sizeof(int4) * (size_t)c->max_work1);

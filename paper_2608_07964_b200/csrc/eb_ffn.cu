@@ -21,13 +21,9 @@
 // the extra rows are never stored), which keeps shared-memory fill traffic close to the weight
 // bytes in the weight-streaming regime.
 //
-// Groups with many rows run on CTA pairs instead (ffn_kernel<PHASE, true>, a 2-CTA cluster): the pair
-// owns a 256-row tile, each CTA loads its own 128 rows of A and one half of the weight tile (for
-// gate/up: CTA 0 the gate rows, CTA 1 the up rows), and the leader CTA issues tcgen05.mma
-// cta_group::2 (M = 256) that reads both halves.  A stage shrinks from 48 KB to 32 KB per CTA for the
-// same tensor-core time, so the ring deepens to 7 stages and L2 traffic per flop drops by a third -
-// that is what the tensor-bound regime needs.  Every CTA fetches its own operands; only the tcgen05.commit
-// that frees a stage is delivered to both CTAs of the pair.
+// Groups of more than 128 rows run on CTA pairs instead (ffn_swap_kernel, a 2-CTA cluster, described at
+// its definition): there the weights are the M = 256 operand of tcgen05.mma cta_group::2 and the token rows
+// are the N operand, so a ragged tile costs the rows it holds (rounded up to 32), not a full tile.
 //
 // Every wait on an mbarrier is bounded: on expiry the kernel records EB_ERR_TIMEOUT in the
 // context status word, lets copies in flight land, frees its TMEM and returns.
@@ -48,13 +44,9 @@ constexpr int kABytes = BM * BK * 2;
 constexpr int kASmallBytes = kSmallRows * BK * 2;
 constexpr int kASlotBytes = kSlotRows * BK * 2;
 constexpr int kBBytes = BN * BK * 2;
-constexpr int kPairStages = 7;
-constexpr int kPairStageBytes = kABytes + kBBytes / 2;   // per CTA of a pair: own A rows + half of B
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 512;
-constexpr size_t kSingleRingBytes = (size_t)kStagesA * kABytes + (size_t)kStagesB * kBBytes;
-constexpr size_t kPairRingBytes = (size_t)kPairStages * kPairStageBytes;
-constexpr size_t kRingBytes = kSingleRingBytes > kPairRingBytes ? kSingleRingBytes : kPairRingBytes;
+constexpr size_t kRingBytes = (size_t)kStagesA * kABytes + (size_t)kStagesB * kBBytes;
 constexpr size_t kSmemBytes = kRingBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 constexpr long long kSpinLimitCycles = 4000000000LL;
@@ -216,8 +208,6 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 }
 // Instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = 256, M = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-// Same with M = 256 for the CTA-pair instruction.
-constexpr uint32_t kIdescPair = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
@@ -227,30 +217,37 @@ __device__ __forceinline__ float silu_mul(uint32_t g_bits, uint32_t u_bits) {
   float g = __uint_as_float(g_bits), u = __uint_as_float(u_bits);
   return __fdividef(g, 1.0f + __expf(-g)) * u;
 }
+// Same value through one special-function instruction instead of two: silu(g) = h + h tanh(h), h = g / 2.
+// tanh.approx.f32 is good to about 2^-11 relative, well inside the bf16 rounding of the result.
+__device__ __forceinline__ float silu_mul_tanh(uint32_t g_bits, uint32_t u_bits) {
+  const float h = 0.5f * __uint_as_float(g_bits), u = __uint_as_float(u_bits);
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(h));
+  return fmaf(h, t, h) * u;
+}
 
 // ---- the grouped GEMM kernel -----------------------------------------------------------------
+// Groups of at most 128 rows, one CTA per 128-row tile.
 // PHASE 1: gate/up + SwiGLU (output 128 columns per tile);  PHASE 2: down (output 256 columns per tile).
-// PAIR false: one CTA per 128-row tile.  PAIR true: a 2-CTA cluster per 256-row tile.
-template <int PHASE, bool PAIR>
+template <int PHASE>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA_small,
            const __grid_constant__ CUtensorMap tmA_slot, const __grid_constant__ CUtensorMap tmB0, const __grid_constant__ CUtensorMap tmB1,
            const int4* __restrict__ work, const int2* __restrict__ slots, const int32_t* __restrict__ work_count,
            bf16* __restrict__ out, int ld_out, int n_out, int k_total, int* status) {
   EB_GRID_DEP_SYNC();
-  // Pair kernel: one ring of kPairStages stages holding {A rows, half of B}.  Single-CTA kernel: two rings,
-  // kStagesA stages of A and kStagesB stages of B, each with its own full/empty barriers, so the weight
-  // copies (DRAM latency) run one k-block further ahead than shared memory would allow with joint stages.
-  constexpr int NA = PAIR ? kPairStages : kStagesA;
-  constexpr int NB = PAIR ? 0 : kStagesB;
+  // Two rings, kStagesA stages of A and kStagesB stages of B, each with its own full/empty barriers, so the
+  // weight copies (DRAM latency) run one k-block further ahead than shared memory would allow with joint stages.
+  constexpr int NA = kStagesA;
+  constexpr int NB = kStagesB;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - raw);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kRingBytes);
   const uint32_t bar0 = base + (uint32_t)kRingBytes;
-  auto a_addr = [&](int s) { return PAIR ? base + s * kPairStageBytes : base + s * kABytes; };
-  auto b_addr = [&](int s) { return PAIR ? base + s * kPairStageBytes + kABytes : base + kStagesA * kABytes + s * kBBytes; };
+  auto a_addr = [&](int s) { return base + s * kABytes; };
+  auto b_addr = [&](int s) { return base + kStagesA * kABytes + s * kBBytes; };
   // barriers: full_a[NA], empty_a[NA], full_b[NB], empty_b[NB], tmem_full[2], tmem_empty[2]
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (NA + s); };
@@ -262,10 +259,9 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
   volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 2 * NA + 2 * NB + 5);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;   // CTA 0 of a pair is the leader
   if (threadIdx.x == 0) {
     for (int s = 0; s < NA; ++s) {
-      mbar_init(full_bar(s), 1);    // producer's arrive + all bytes of the stage (pair: of both CTAs, leader only)
+      mbar_init(full_bar(s), 1);    // producer's arrive + all bytes of the stage
       mbar_init(empty_bar(s), 1);   // one tcgen05.commit
     }
     for (int s = 0; s < NB; ++s) {
@@ -274,34 +270,27 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);                // one tcgen05.commit
-      mbar_init(tempty_bar(a), PAIR ? 8 : 4);    // one arrival per epilogue warp (pair: of both CTAs, leader only)
+      mbar_init(tempty_bar(a), 4);               // one arrival per epilogue warp
     }
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     prefetch_tmap(&tmA);
-    if (!PAIR) prefetch_tmap(&tmA_small);
-    if (!PAIR) prefetch_tmap(&tmA_slot);
+    prefetch_tmap(&tmA_small);
+    prefetch_tmap(&tmA_slot);
     prefetch_tmap(&tmB0);
     if (PHASE == 1) prefetch_tmap(&tmB1);
   }
   if (warp == 1) {
-    if (PAIR) {
-      tmem_alloc_pair(smem_u32((const void*)s_tmem), kTmemCols);
-      tmem_relinquish_pair();
-    } else {
-      tmem_alloc(smem_u32((const void*)s_tmem), kTmemCols);
-      tmem_relinquish();
-    }
+    tmem_alloc(smem_u32((const void*)s_tmem), kTmemCols);
+    tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
-  if (PAIR) cluster_sync_all();   // the peer's barriers are initialised before anything arrives on them
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
-  const int n_work = work_count[(PAIR ? 5 : 0) + PHASE - 1];
+  const int n_work = work_count[PHASE - 1];
   const int num_kb = (k_total + BK - 1) / BK;
-  const int w_first = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
-  const int w_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+  const int w_first = (int)blockIdx.x, w_step = (int)gridDim.x;
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -312,13 +301,13 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
         // x = first row, y = valid rows, z = weight matrix, w = n tile; y < 0 marks a merged tile:
         // (-y & 15) slots of 16 rows each, or of 32 rows each if (-y & 16), described by slots[x ..)
         const int4 it = __ldg(work + w);
-        const bool merged = !PAIR && it.y < 0;
+        const bool merged = it.y < 0;
         const int n_slots = merged ? ((-it.y) & 15) : 0;
         const bool big_slots = merged && ((-it.y) & 16);
         int slot_row[kMergeSlots];
 #pragma unroll
         for (int i = 0; i < kMergeSlots; ++i) slot_row[i] = (merged && i < n_slots) ? __ldg(slots + it.x + i).x : 0;
-        const bool small = !PAIR && !merged && it.y <= kSmallRows;
+        const bool small = !merged && it.y <= kSmallRows;
         const uint32_t tx_a = (uint32_t)(merged ? n_slots * (big_slots ? kASmallBytes : kASlotBytes) : small ? kASmallBytes : kABytes);
         // One specialised k loop per tile kind, so the issuing thread does the minimum between a stage
         // becoming free and its copies being in flight (that delay comes straight off the prefetch depth).
@@ -348,19 +337,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
     stage = 0;              \
     phase ^= 1u;            \
   }
-        if (PAIR) {
-          const CUtensorMap* bmap = (PHASE == 1 && rank == 1) ? &tmB1 : &tmB0;
-          const int brow = PHASE == 1 ? it.w * 128 : it.w * BN + (int)rank * 128;
-          for (int kb = 0; kb < num_kb; ++kb) {
-            EB_A_STAGE_BEGIN();
-            // both CTAs' copies are counted on the leader's barrier; the leader announces the total
-            const uint32_t fb = map_to_cta(full_bar(stage), 0);
-            if (rank == 0) mbar_expect_tx(full_bar(stage), 2u * kPairStageBytes);
-            tma_pair_load_2d(sa, &tmA, kb * BK, it.x + (int)rank * BM, fb);
-            tma_pair_load_3d(b_addr(stage), bmap, kb * BK, brow, it.z, fb);
-            EB_A_STAGE_END();
-          }
-        } else if (!merged) {
+        if (!merged) {
           const CUtensorMap* amap = small ? &tmA_small : &tmA;
           for (int kb = 0; kb < num_kb; ++kb) {
             EB_B_STAGE();
@@ -396,8 +373,8 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer (pair: leader CTA only) ----------------
-    if (lane == 0 && rank == 0) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
       int stage = 0, stage_b = 0;
       uint32_t phase = 0, phase_b = 0;
       int local = 0;
@@ -409,24 +386,17 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
         const uint32_t d_tmem = tmem_base + as * BN;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, s_abort, status)) goto done;
-          if (!PAIR && !mbar_wait(fullb_bar(stage_b), phase_b, s_abort, status)) goto done;
+          if (!mbar_wait(fullb_bar(stage_b), phase_b, s_abort, status)) goto done;
           tc_fence_after();
-          const uint64_t da = smem_desc(a_addr(stage)), db = smem_desc(b_addr(PAIR ? stage : stage_b));
+          const uint64_t da = smem_desc(a_addr(stage)), db = smem_desc(b_addr(stage_b));
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k) {
-            if (PAIR) umma_pair_bf16(d_tmem, da + 2 * k, db + 2 * k, kIdescPair, (kb | k) != 0 ? 1u : 0u);
-            else umma_bf16(d_tmem, da + 2 * k, db + 2 * k, kIdesc, (kb | k) != 0 ? 1u : 0u);
-          }
-          // the stages are reusable (in both CTAs of a pair) once these MMAs have read them
-          if (PAIR) {
-            umma_pair_commit(empty_bar(stage));
-          } else {
-            umma_commit(empty_bar(stage));
-            umma_commit(emptyb_bar(stage_b));
-            if (++stage_b == kStagesB) {
-              stage_b = 0;
-              phase_b ^= 1u;
-            }
+          for (int k = 0; k < BK / 16; ++k) umma_bf16(d_tmem, da + 2 * k, db + 2 * k, kIdesc, (kb | k) != 0 ? 1u : 0u);
+          // the stages are reusable once these MMAs have read them
+          umma_commit(empty_bar(stage));
+          umma_commit(emptyb_bar(stage_b));
+          if (++stage_b == kStagesB) {
+            stage_b = 0;
+            phase_b ^= 1u;
           }
           if (++stage == NA) {
             stage = 0;
@@ -434,7 +404,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
           }
         }
         // accumulator complete
-        if (PAIR) umma_pair_commit(tfull_bar(as)); else umma_commit(tfull_bar(as));
+        umma_commit(tfull_bar(as));
       }
     }
   } else {
@@ -445,12 +415,16 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
       const int4 it = __ldg(work + w);
       const int as = local & 1;
       const uint32_t aphase = (local >> 1) & 1u;
-      if (!mbar_wait(tfull_bar(as), aphase, s_abort, status)) goto done;
+      // one lane waits, the outcome is made warp-uniform before any .aligned instruction
+      int ok = 1;
+      if (lane == 0) ok = mbar_wait(tfull_bar(as), aphase, s_abort, status) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) goto done;
       tc_fence_after();
-      int r = (int)rank * BM + q * 32 + lane;   // row inside the (pair's) tile
+      int r = q * 32 + lane;                    // row inside the tile
       bool row_ok = r < it.y;
       int row_g = it.x + r;                     // row in the permuted order
-      if (!PAIR && it.y < 0) {
+      if (it.y < 0) {
         // merged tile: epilogue warp q owns slot q (32-row slots) or slots 2q and 2q+1 (16-row slots)
         row_ok = false;
         const int v = -it.y;
@@ -519,10 +493,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
       // all TMEM reads of this warp are complete (wait::ld above): hand the accumulator back
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) {
-        if (PAIR) mbar_arrive_cluster(map_to_cta(tempty_bar(as), 0));
-        else mbar_arrive(tempty_bar(as));
-      }
+      if (lane == 0) mbar_arrive(tempty_bar(as));
     }
   }
 
@@ -533,10 +504,246 @@ done:
   }
   tc_fence_before();
   __syncthreads();
-  if (PAIR) cluster_sync_all();   // neither CTA leaves while its peer may still touch its memory or barriers
   if (warp == 1) {
     tc_fence_after();
-    if (PAIR) tmem_dealloc_pair(tmem_base, kTmemCols); else tmem_dealloc(tmem_base, kTmemCols);
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---- CTA-pair kernel with the weights as the M operand ------------------------------------------
+// Groups of more than 128 rows.  The pair's M = 256 rows are weight rows (128 per CTA) and the
+// accumulator columns are token rows: N = the tile's valid rows rounded up to 32 (at most 256), so the
+// tensor-core work of a ragged tile is what it holds, not a full 256-row tile.  Every k-step issues
+// two MMAs that share the token operand:
+//   gate/up: W0 = 256 rows of W_gate, W1 = the same 256 rows of W_up; the lane that holds gate output i
+//            holds up output i of the same token, so SiLU * up fuses in registers (256 outputs per tile);
+//   down   : W0, W1 = two consecutive 256-row blocks of W_down (512 outputs per tile).
+// A stage is 48 KB per CTA (2 x 128 weight rows + up to 128 token rows of one k-block) for up to 1024
+// tensor-core cycles: a quarter less shared-memory fill per flop than 256 x 256 tiles.  The two
+// accumulators fill TMEM (2 x 256 columns), so the epilogue of a tile does not overlap the next tile's
+// MMAs; eight epilogue warps (two per TMEM lane quadrant, alternating 16-column chunks) keep that gap
+// short, and the producer keeps prefetching through it.  The accumulator holds outputs in lanes and
+// tokens in columns: a warp stores 32 consecutive outputs of one token (64 bytes) per instruction.
+constexpr int kSwStages = 4;
+constexpr int kSwWBytes = 128 * BK * 2;                        // 128 weight rows of one k-block
+constexpr int kSwStageBytes = 2 * kSwWBytes + kABytes;         // W0 | W1 | token rows
+constexpr int kSwRingBytes = kSwStages * kSwStageBytes;
+constexpr int kSwEpiWarps = 8;
+constexpr size_t kSwSmemBytes = (size_t)kSwRingBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + kSwEpiWarps * 2048 /*transposes*/;
+static_assert(kSwSmemBytes <= 232448, "shared memory of one CTA");
+constexpr int kSwThreads = 64 + 32 * kSwEpiWarps;
+constexpr int kSwTileRows = 256;                               // token rows of a tile at most
+constexpr int kSwFeat1 = 256;                                  // outputs of a gate/up tile
+constexpr int kSwFeat2 = 512;                                  // outputs of a down tile
+constexpr uint32_t kIdescSwBase = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 4) << 24);
+
+__device__ __forceinline__ int sw_cols(int valid_rows) {
+  const int n = (valid_rows + 31) & ~31;
+  return n > kSwTileRows ? kSwTileRows : n;
+}
+
+template <int PHASE>
+__global__ void __launch_bounds__(kSwThreads, 1)
+ffn_swap_kernel(const __grid_constant__ CUtensorMap tmT128, const __grid_constant__ CUtensorMap tmT64,
+                const __grid_constant__ CUtensorMap tmT32, const __grid_constant__ CUtensorMap tmT16,
+                const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
+                const int4* __restrict__ work, const int32_t* __restrict__ work_count, bf16* __restrict__ out,
+                int ld_out, int n_out, int k_total, int* status) {
+  EB_GRID_DEP_SYNC();
+  constexpr int NS = kSwStages;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kSwRingBytes);
+  const uint32_t bar0 = base + (uint32_t)kSwRingBytes;
+  auto w0_addr = [&](int s) { return base + s * kSwStageBytes; };
+  auto w1_addr = [&](int s) { return base + s * kSwStageBytes + kSwWBytes; };
+  auto t_addr = [&](int s) { return base + s * kSwStageBytes + 2 * kSwWBytes; };
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (NS + s); };
+  const uint32_t tfull_bar = bar0 + 8u * (2 * NS), tempty_bar = bar0 + 8u * (2 * NS + 1);
+  volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(bars + 2 * NS + 2);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 2 * NS + 3);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();   // CTA 0 of a pair is the leader
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < NS; ++s) {
+      mbar_init(full_bar(s), 1);    // the leader's arrive + all bytes of the stage of both CTAs
+      mbar_init(empty_bar(s), 1);   // one tcgen05.commit (delivered to both CTAs)
+    }
+    mbar_init(tfull_bar, 1);                  // one tcgen05.commit
+    mbar_init(tempty_bar, 2 * kSwEpiWarps);   // one arrival per epilogue warp of both CTAs (leader's barrier)
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    prefetch_tmap(&tmT128);
+    prefetch_tmap(&tmT64);
+    prefetch_tmap(&tmT32);
+    prefetch_tmap(&tmT16);
+    prefetch_tmap(&tmW0);
+    prefetch_tmap(&tmW1);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32((const void*)s_tmem), kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();   // the peer's barriers are initialised before anything arrives on them
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+  const int n_work = work_count[5 + PHASE - 1];
+  const int num_kb = (k_total + BK - 1) / BK;
+  // The list is ordered by cost, widest tiles first.  It is dealt out in rounds of one tile per pair, the
+  // direction alternating from round to round, so every pair ends up with nearly the same total cost.
+  const int n_pairs = (int)(gridDim.x >> 1), my_pair = (int)(blockIdx.x >> 1);
+  auto tile_of_round = [&](int r) { return r * n_pairs + ((r & 1) ? n_pairs - 1 - my_pair : my_pair); };
+
+  if (warp == 0) {
+    // ---------------- TMA producer (each CTA loads its own halves) ----------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int r = 0; r * n_pairs < n_work; ++r) {
+        const int w = tile_of_round(r);
+        if (w >= n_work) continue;
+        const int4 it = __ldg(work + w);   // x = first row, y = valid rows, z = weight matrix, w = output tile
+        const int half = sw_cols(it.y) >> 1;            // token rows this CTA loads: a multiple of 16
+        const int tok0 = it.x + (int)rank * half;
+        const int wrow0 = PHASE == 1 ? it.w * kSwFeat1 + (int)rank * 128 : it.w * kSwFeat2 + (int)rank * 128;
+        const int wrow1 = PHASE == 1 ? wrow0 : wrow0 + 256;
+        const uint32_t tx = 2u * (2u * kSwWBytes + (uint32_t)half * (BK * 2));
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, s_abort, status)) goto done;
+          // both CTAs' copies are counted on the leader's barrier; the leader announces the total
+          const uint32_t fb = map_to_cta(full_bar(stage), 0);
+          if (rank == 0) mbar_expect_tx(full_bar(stage), tx);
+          tma_pair_load_3d(w0_addr(stage), &tmW0, kb * BK, wrow0, it.z, fb);
+          tma_pair_load_3d(w1_addr(stage), &tmW1, kb * BK, wrow1, it.z, fb);
+          const uint32_t ta = t_addr(stage);
+          if (half == 128) {
+            tma_pair_load_2d(ta, &tmT128, kb * BK, tok0, fb);
+          } else {
+            int r = 0;   // rows placed so far; every box starts on a multiple of 16 rows (2 KB), which keeps the swizzle phase
+            if (half & 64) {
+              tma_pair_load_2d(ta, &tmT64, kb * BK, tok0, fb);
+              r = 64;
+            }
+            if (half & 32) {
+              tma_pair_load_2d(ta + r * (BK * 2), &tmT32, kb * BK, tok0 + r, fb);
+              r += 32;
+            }
+            if (half & 16) tma_pair_load_2d(ta + r * (BK * 2), &tmT16, kb * BK, tok0 + r, fb);
+          }
+          if (++stage == NS) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer (leader CTA only) ----------------
+    if (lane == 0 && rank == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int local = -1;
+      for (int r = 0; r * n_pairs < n_work; ++r) {
+        const int w = tile_of_round(r);
+        if (w >= n_work) continue;
+        ++local;
+        const int4 it = __ldg(work + w);
+        const uint32_t idesc = kIdescSwBase | ((uint32_t)(sw_cols(it.y) >> 3) << 17);
+        if (!mbar_wait(tempty_bar, (uint32_t)(local & 1) ^ 1u, s_abort, status)) goto done;
+        tc_fence_after();
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, s_abort, status)) goto done;
+          tc_fence_after();
+          const uint64_t d0 = smem_desc(w0_addr(stage)), d1 = smem_desc(w1_addr(stage)), dt = smem_desc(t_addr(stage));
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            umma_pair_bf16(tmem_base, d0 + 2 * k, dt + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            umma_pair_bf16(tmem_base + 256, d1 + 2 * k, dt + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_pair_commit(empty_bar(stage));   // the stage is reusable in both CTAs once these MMAs have read it
+          if (++stage == NS) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+        umma_pair_commit(tfull_bar);   // both accumulators complete
+      }
+    }
+  } else {
+    // ---------------- epilogue warps ----------------
+    const int q = warp & 3;                 // TMEM lane quadrant this warp may read
+    const int chunk0 = ((warp - 2) >> 2) * 16;   // the two warps of a quadrant take alternate 16-column chunks
+    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+    bf16* tile = reinterpret_cast<bf16*>(smem + kSwRingBytes + 256) + (warp - 2) * 1024;   // 2 KB per epilogue warp
+    int local = -1;
+    for (int r = 0; r * n_pairs < n_work; ++r) {
+      const int w = tile_of_round(r);
+      if (w >= n_work) continue;
+      ++local;
+      const int4 it = __ldg(work + w);
+      // one lane waits, the outcome is made warp-uniform before any .aligned instruction
+      int ok = 1;
+      if (lane == 0) ok = mbar_wait(tfull_bar, (uint32_t)(local & 1), s_abort, status) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) goto done;
+      tc_fence_after();
+      // this warp's 32 outputs start at fbase; a 16-token chunk is transposed through shared memory so that
+      // global stores are 16-byte vectors: lane -> (token lane / 4 (+8), outputs 8 (lane % 4) .. +7)
+      const int fbase = (PHASE == 1 ? it.w * kSwFeat1 : it.w * kSwFeat2) + (int)rank * 128 + q * 32;
+      const int fcol = fbase + (lane & 3) * 8;
+#pragma unroll 1
+      for (int c0 = chunk0; c0 < it.y; c0 += 32) {
+        uint32_t a[16], b[16];
+        tmem_ld16(taddr + c0, a);
+        tmem_ld16(taddr + 256 + c0, b);
+        tmem_ld_wait();
+        if (PHASE == 1) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) tile[j * 32 + lane] = __float2bfloat16_rn(silu_mul_tanh(a[j], b[j]));
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            tile[j * 32 + lane] = __float2bfloat16_rn(__uint_as_float(a[j]));
+            tile[512 + j * 32 + lane] = __float2bfloat16_rn(__uint_as_float(b[j]));
+          }
+        }
+        __syncwarp();
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          const int tok = (lane >> 2) + 8 * r;
+          if (c0 + tok < it.y) {
+            bf16* dst = out + (size_t)(it.x + c0 + tok) * ld_out + fcol;
+            const uint4* src = reinterpret_cast<const uint4*>(tile + tok * 32 + (lane & 3) * 8);
+            if (fcol < n_out) *reinterpret_cast<uint4*>(dst) = src[0];
+            if (PHASE == 2 && fcol + 256 < n_out) *reinterpret_cast<uint4*>(dst + 256) = src[64];   // second tile: +512 bf16
+          }
+        }
+        __syncwarp();
+      }
+      // all TMEM reads of this warp are complete (wait::ld above): hand the accumulators back
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar, 0));
+    }
+  }
+
+done:
+  if (*s_abort) {
+    // give copies and MMAs in flight time to land before shared memory and TMEM go away
+    for (int i = 0; i < 200; ++i) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();   // neither CTA leaves while its peer may still touch its memory or barriers
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
   }
 }
 
@@ -559,13 +766,12 @@ __global__ void bounded_wait_probe_kernel(long long limit_cycles, int* status, i
 }
 
 // ---- tile list construction ------------------------------------------------------------------
-// A group runs either on single CTAs (128-row tiles) or on CTA pairs (256-row tiles), never both, so
-// its weights are streamed by one kernel only.  Pairs are used when they do not add padded rows
-// compared with 128-row tiles, or when the group is large enough for the padding not to matter.
-__device__ __forceinline__ bool group_uses_pairs(int rows) {
-  const int rem = rows % (2 * BM);
-  return rows > BM && (rows >= 4 * BM || rem == 0 || rem > BM);
-}
+// A group runs either on single CTAs (128-row tiles: groups of at most 128 rows) or on CTA pairs (the
+// kernel with the weights as the M operand: everything larger), never both, so its weights are streamed
+// by one kernel only.  A pair group of `rows` rows is cut into ceil(rows / 256) tiles of nearly equal
+// size, so no tile is a short remainder that would still stream a whole weight tile.
+__device__ __forceinline__ bool group_uses_pairs(int rows) { return rows > BM; }
+__device__ __forceinline__ int pair_tiles(int rows) { return (rows + kSwTileRows - 1) / kSwTileRows; }
 
 // Processing order of the groups.  The group table is device-major, so the D replicas of a shared
 // expert (one group per virtual device, all reading the same weight matrix) lie far apart in it.
@@ -613,31 +819,70 @@ __device__ __forceinline__ bool merged_class(const ModelParams& mp, const int* d
   return mx <= kMergeMaxRows;
 }
 
-// plan: per group (in processing order) of the requested range, number of 128-row tiles or of 256-row
-// pair tiles; exclusive scans of both; totals.
+// Block-wide exclusive scan of one value per thread (1024 threads); returns the exclusive prefix and
+// leaves the block total in *total.  Ends with a barrier, so s_warp may be reused right away.
+__device__ __forceinline__ long long block_scan_excl(long long v, long long* s_warp, long long* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  long long incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    long long n = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += n;
+  }
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    long long wv = s_warp[lane], wi = wv;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      long long n = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += n;
+    }
+    s_warp[lane] = wi - wv;
+    if (lane == 31) s_warp[32] = wi;
+  }
+  __syncthreads();
+  const long long excl = s_warp[warp] + incl - v;
+  *total = s_warp[32];
+  __syncthreads();
+  return excl;
+}
+
+// Columns (token rows rounded up to 32) of the largest tile of a pair group: its cost class.
+__device__ __forceinline__ int pair_group_cols(int rows) {
+  const int t = pair_tiles(rows);
+  return sw_cols((rows + t - 1) / t);
+}
+
+// plan: per group (in processing order) of the requested range, its number of 128-row tiles (single-CTA
+// lists) with an exclusive scan; the pair groups (more than 128 rows) are listed separately, ordered by
+// the cost of their tiles (widest first, table order inside a cost class), with the scan of their tile
+// counts.  Widest-first order lets the pair kernel deal its tiles out in rounds of near-equal cost.
 __global__ void __launch_bounds__(1024)
 plan_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t* __restrict__ step_meta, int device,
-            int nt1, int nt2, int pair_mode, int32_t* __restrict__ mtile_pref, int32_t* __restrict__ ptile_pref,
-            int32_t* __restrict__ pgroup, int32_t* __restrict__ pchunks, int32_t* __restrict__ work_count) {
+            int nt1, int nt2, int nt1p, int nt2p, int pair_mode, int32_t* __restrict__ mtile_pref,
+            int32_t* __restrict__ ptile_pref, int32_t* __restrict__ pgroup, int32_t* __restrict__ ppgroup,
+            int32_t* __restrict__ pchunks, int32_t* __restrict__ work_count) {
   EB_GRID_DEP_SYNC();
-  __shared__ long long s_warp[32];
-  __shared__ long long s_carry;
+  __shared__ long long s_warp[33];
   __shared__ int s_dev_off[EB_MAX_D + 1];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x;
   if (tid <= mp.D) s_dev_off[tid] = mp.dev_off[tid];
   const int G = step_meta[1];
   const int g0 = device < 0 ? 0 : step_meta[3 + device];
   const int g1 = device < 0 ? G : step_meta[3 + device + 1];
   const int ng = g1 - g0;
   const int nl = step_meta[2];
-  if (tid == 0) s_carry = 0;
   __syncthreads();
+  long long carry = 0;      // single tiles so far
+  int any_pairs = 0;
   for (int b = 0; b < ng; b += 1024) {
-    int i = b + tid;
-    long long v = 0;  // low 32 bits: single tiles, high 32 bits: pair tiles
+    const int i = b + tid;
+    long long v = 0;
+    int is_pair = 0;
     if (i < ng) {
       const int g = group_at(mp, s_dev_off, nl, device, g0, i);
-      int rows = group_off[g + 1] - group_off[g];
+      const int rows = group_off[g + 1] - group_off[g];
       int head, chunks;
       pgroup[i] = g;
       pchunks[i] = -1;
@@ -646,42 +891,46 @@ plan_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t
         v = i == head ? ((chunks & 0xffff) + per_tile - 1) / per_tile : 0;   // the class's tiles sit at its first position
         pchunks[i] = chunks;
       } else if (pair_mode && group_uses_pairs(rows)) {
-        v = (long long)((rows + 2 * BM - 1) / (2 * BM)) << 32;
+        is_pair = 1;
       } else {
         v = (rows + BM - 1) / BM;
       }
     }
-    long long incl = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      long long n = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += n;
-    }
-    if (lane == 31) s_warp[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-      long long wv = s_warp[lane], wi = wv;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        long long n = __shfl_up_sync(0xffffffffu, wi, o);
-        if (lane >= o) wi += n;
+    long long total;
+    const long long excl = block_scan_excl(v, s_warp, &total);
+    if (i < ng) mtile_pref[i] = (int)(carry + excl);
+    carry += total;
+    any_pairs |= __syncthreads_or(is_pair);
+  }
+  long long pcarry = 0;   // low 32 bits: pair groups listed so far, high 32 bits: their tiles
+  if (any_pairs) {
+    for (int cols = kSwTileRows; cols >= 32; cols -= 32) {
+      for (int b = 0; b < ng; b += 1024) {
+        const int i = b + tid;
+        long long v = 0;
+        int g = 0;
+        if (i < ng) {
+          g = pgroup[i];
+          const int rows = group_off[g + 1] - group_off[g];
+          if (pchunks[i] < 0 && group_uses_pairs(rows) && pair_group_cols(rows) == cols)
+            v = 1LL | ((long long)pair_tiles(rows) << 32);
+        }
+        if (!__syncthreads_or(v != 0)) continue;
+        long long total;
+        const long long excl = block_scan_excl(v, s_warp, &total);
+        if (v) {
+          const long long at = pcarry + excl;
+          ppgroup[(int)(at & 0xffffffffLL)] = g;
+          ptile_pref[(int)(at & 0xffffffffLL)] = (int)(at >> 32);
+        }
+        pcarry += total;
       }
-      s_warp[lane] = wi - wv;
     }
-    __syncthreads();
-    long long excl = s_carry + s_warp[warp] + incl - v;
-    if (i < ng) {
-      mtile_pref[i] = (int)(excl & 0xffffffffLL);
-      ptile_pref[i] = (int)(excl >> 32);
-    }
-    __syncthreads();
-    if (tid == 1023) s_carry = excl + v;
-    __syncthreads();
   }
   if (tid == 0) {
-    const int mt = (int)(s_carry & 0xffffffffLL), pt = (int)(s_carry >> 32);
+    const int mt = (int)carry, npg = (int)(pcarry & 0xffffffffLL), pt = (int)(pcarry >> 32);
     mtile_pref[ng] = mt;
-    ptile_pref[ng] = pt;
+    ptile_pref[npg] = pt;
     work_count[0] = mt * nt1;
     work_count[1] = mt * nt2;
     work_count[2] = mt;
@@ -689,9 +938,10 @@ plan_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t
     work_count[4] = ng;
     work_count[8] = nl;
     work_count[9] = device;
-    work_count[5] = pt * nt1;
-    work_count[6] = pt * nt2;
+    work_count[5] = pt * nt1p;
+    work_count[6] = pt * nt2p;
     work_count[7] = pt;
+    work_count[10] = npg;
   }
 }
 
@@ -700,25 +950,25 @@ plan_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t
 __global__ void __launch_bounds__(256)
 fill_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t* __restrict__ group_w,
             const int32_t* __restrict__ mtile_pref, const int32_t* __restrict__ ptile_pref,
-            const int32_t* __restrict__ pgroup, const int32_t* __restrict__ pchunks,
-            const int32_t* __restrict__ work_count, int nt1, int nt2, int max1, int max2, int maxp1, int maxp2,
+            const int32_t* __restrict__ pgroup, const int32_t* __restrict__ ppgroup, const int32_t* __restrict__ pchunks,
+            const int32_t* __restrict__ work_count, int nt1, int nt2, int nt1p, int nt2p, int max1, int max2,
+            int maxp1, int maxp2,
             int4* __restrict__ work1, int4* __restrict__ work2, int4* __restrict__ work1p, int4* __restrict__ work2p,
             int2* __restrict__ slots) {
   EB_GRID_DEP_SYNC();
-  const int ng = work_count[4];
+  const int ng = work_count[4], npg = work_count[10];
   const int cnt[4] = {work_count[0], work_count[1], work_count[5], work_count[6]};
   const int total = cnt[0] + cnt[1] + cnt[2] + cnt[3];
   for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
     int list = 0, local = idx;
     while (local >= cnt[list]) local -= cnt[list++];
     const bool pair = list >= 2;
-    const int nt = (list & 1) ? nt2 : nt1;
-    const int tile_rows = pair ? 2 * BM : BM;
+    const int nt = pair ? ((list & 1) ? nt2p : nt1p) : ((list & 1) ? nt2 : nt1);
     const int32_t* pref = pair ? ptile_pref : mtile_pref;
     const int t_index = local / nt;
     // largest gi with pref[gi] <= t_index: groups without tiles in this list share their successor's
     // prefix, and a group that owns tiles has pref[gi + 1] > pref[gi]
-    int lo = 0, hi = ng - 1;
+    int lo = 0, hi = (pair ? npg : ng) - 1;
     while (lo < hi) {
       int mid = (lo + hi + 1) >> 1;
       if (pref[mid] <= t_index) lo = mid; else hi = mid - 1;
@@ -727,9 +977,9 @@ fill_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t
     const int t_g = pref[gi + 1] - pref[gi];
     const int rem = local - pref[gi] * nt;
     const int n = rem / t_g, m = rem % t_g;
-    const int g = pgroup[gi];
+    const int g = pair ? ppgroup[gi] : pgroup[gi];
     int4 it;
-    const int head = gi, chunks_raw = pchunks[gi];   // only the first position of a merged class owns tiles
+    const int head = gi, chunks_raw = pair ? -1 : pchunks[gi];   // only the first position of a merged class owns tiles
     if (!pair && chunks_raw >= 0) {
       // tile m of a merged class holds the next 8 (16-row) or 4 (32-row) chunks of the class, replicas in
       // device order
@@ -751,10 +1001,16 @@ fill_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t
       }
       it.x = base;
       it.y = -(n_here | (big ? 16 : 0));
+    } else if (pair) {
+      // t_g tiles of nearly equal size: the first (rows % t_g) tiles hold one row more
+      const int rows = group_off[g + 1] - group_off[g];
+      const int each = rows / t_g, more = rows % t_g;
+      it.x = group_off[g] + m * each + min(m, more);
+      it.y = each + (m < more ? 1 : 0);
     } else {
-      const int row0 = group_off[g] + m * tile_rows;
+      const int row0 = group_off[g] + m * BM;
       it.x = row0;
-      it.y = min(tile_rows, group_off[g + 1] - row0);
+      it.y = min(BM, group_off[g + 1] - row0);
     }
     it.z = group_w[g];
     it.w = n;
@@ -796,19 +1052,19 @@ bool make_map(CUtensorMap* m, const void* ptr, uint64_t d0, uint64_t d1, uint64_
   return r == CUDA_SUCCESS;
 }
 
-template <int PHASE, bool PAIR>
+template <int PHASE>
 cudaError_t launch_ffn(eb_ctx* c, cudaStream_t st, const CUtensorMap& tA, const CUtensorMap& tAs, const CUtensorMap& tB0,
                        const CUtensorMap& tB1, const int4* work, bf16* out, int ld_out, int n_out, int k_total,
                        const CUtensorMap& tAslot) {
   const int2* slots = c->slots;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(PAIR ? c->pair_grid : c->num_sms);
+  cfg.gridDim = dim3(c->num_sms);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+  attr[0].val.clusterDim.x = 1;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -817,8 +1073,31 @@ cudaError_t launch_ffn(eb_ctx* c, cudaStream_t st, const CUtensorMap& tA, const 
   cfg.numAttrs = 2;
   const int32_t* wc = c->work_count;
   ++g_ebi_launches;
-  return cudaLaunchKernelEx(&cfg, ffn_kernel<PHASE, PAIR>, tA, tAs, tAslot, tB0, tB1, work, slots, wc, out, ld_out, n_out, k_total,
+  return cudaLaunchKernelEx(&cfg, ffn_kernel<PHASE>, tA, tAs, tAslot, tB0, tB1, work, slots, wc, out, ld_out, n_out, k_total,
                             c->d_status);
+}
+
+template <int PHASE>
+cudaError_t launch_swap(eb_ctx* c, cudaStream_t st, const CUtensorMap* tT, const CUtensorMap& tW0, const CUtensorMap& tW1,
+                        const int4* work, bf16* out, int ld_out, int n_out, int k_total) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(c->pair_grid);
+  cfg.blockDim = dim3(kSwThreads);
+  cfg.dynamicSmemBytes = kSwSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  const int32_t* wc = c->work_count;
+  ++g_ebi_launches;
+  return cudaLaunchKernelEx(&cfg, ffn_swap_kernel<PHASE>, tT[0], tT[1], tT[2], tT[3], tW0, tW1, work, wc, out, ld_out, n_out,
+                            k_total, c->d_status);
 }
 
 }  // namespace
@@ -840,16 +1119,16 @@ eb_status ebi_ffn_bind(eb_ctx* c) {
     return ebi_fail(c, EB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the weights");
   int pair_grid = 0;
   {   // per context: function attributes and cluster occupancy belong to the current device
-    cudaError_t e = cudaFuncSetAttribute(ffn_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(ffn_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_swap_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSwSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_swap_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSwSmemBytes);
     if (e != cudaSuccess) return ebi_check_cuda(c, e, "cudaFuncSetAttribute");
     // how many 2-CTA clusters of this kernel the device can hold at once (one CTA per SM)
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * (c->num_sms / 2));
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.blockDim = dim3(kSwThreads);
+    cfg.dynamicSmemBytes = kSwSmemBytes;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
@@ -858,7 +1137,7 @@ eb_status ebi_ffn_bind(eb_ctx* c) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int clusters = 0;
-    e = cudaOccupancyMaxActiveClusters(&clusters, ffn_kernel<1, true>, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&clusters, ffn_swap_kernel<1>, &cfg);
     if (e != cudaSuccess || clusters < 1) {
       cudaGetLastError();
       clusters = 0;   // pairs unavailable: every group runs on single CTAs
@@ -878,44 +1157,48 @@ eb_status ebi_ffn_run(eb_ctx* c, cudaStream_t st, const void* xp, const int32_t*
   if (!c->ws) return ebi_fail(c, EB_ERR_WORKSPACE, "no workspace set");
   const eb_config& g = c->cfg;
   const int rows = ebi_rows_cap(c);
-  CUtensorMap tm_x, tm_xs, tm_xl, tm_a, tm_as, tm_al;
+  CUtensorMap tm_x, tm_xs, tm_xl, tm_a, tm_as, tm_al, tm_x64, tm_a64;
   if (!make_map(&tm_x, xp, g.H, rows, 0, BK, BM) || !make_map(&tm_xs, xp, g.H, rows, 0, BK, kSmallRows) ||
       !make_map(&tm_xl, xp, g.H, rows, 0, BK, kSlotRows) || !make_map(&tm_a, c->act, g.I, rows, 0, BK, BM) ||
-      !make_map(&tm_as, c->act, g.I, rows, 0, BK, kSmallRows) || !make_map(&tm_al, c->act, g.I, rows, 0, BK, kSlotRows))
+      !make_map(&tm_as, c->act, g.I, rows, 0, BK, kSmallRows) || !make_map(&tm_al, c->act, g.I, rows, 0, BK, kSlotRows) ||
+      !make_map(&tm_x64, xp, g.H, rows, 0, BK, 64) || !make_map(&tm_a64, c->act, g.I, rows, 0, BK, 64))
     return ebi_fail(c, EB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the activations");
+  // token-row boxes of 128 / 64 / 32 / 16 rows for the pair kernel
+  const CUtensorMap tok_x[4] = {tm_x, tm_x64, tm_xs, tm_xl}, tok_a[4] = {tm_a, tm_a64, tm_as, tm_al};
   const int nt1 = (g.I + 127) / 128, nt2 = (g.H + BN - 1) / BN;
+  const int nt1p = (g.I + kSwFeat1 - 1) / kSwFeat1, nt2p = (g.H + kSwFeat2 - 1) / kSwFeat2;
   // CTA pairs only pay for groups of more than 128 rows; skip their launches when the permutation that
   // produced this step (same step_meta buffer) says no group can be that large
   bool pairs = c->pair_grid >= 2 && c->cfg.max_tokens > BM;
   if (pairs && c->hint_meta == step_meta && c->hint_max_group_rows >= 0 && c->hint_max_group_rows <= BM) pairs = false;
   {
     KernelTimer timer(c, EBK_FFN_PLAN, st);
-    ebi_launch(plan_kernel, dim3(1), dim3(1024), 0, st, c->mp, group_off, step_meta, (int)device, nt1, nt2, pairs ? 1 : 0,
-               c->mtile_pref, c->ptile_pref, c->pgroup, c->pchunks, c->work_count);
+    ebi_launch(plan_kernel, dim3(1), dim3(1024), 0, st, c->mp, group_off, step_meta, (int)device, nt1, nt2, nt1p, nt2p, pairs ? 1 : 0,
+               c->mtile_pref, c->ptile_pref, c->pgroup, c->ppgroup, c->pchunks, c->work_count);
   }
   {
     KernelTimer timer(c, EBK_FFN_FILL, st);
     ebi_launch(fill_kernel, dim3(c->num_sms), dim3(256), 0, st, c->mp, group_off, group_w, (const int32_t*)c->mtile_pref,
-               (const int32_t*)c->ptile_pref, (const int32_t*)c->pgroup, (const int32_t*)c->pchunks,
-               (const int32_t*)c->work_count, nt1, nt2, c->max_work1, c->max_work2,
+               (const int32_t*)c->ptile_pref, (const int32_t*)c->pgroup, (const int32_t*)c->ppgroup, (const int32_t*)c->pchunks,
+               (const int32_t*)c->work_count, nt1, nt2, nt1p, nt2p, c->max_work1, c->max_work2,
                c->max_work1p, c->max_work2p, c->work1, c->work2, c->work1p, c->work2p, c->slots);
   }
   cudaError_t e = cudaSuccess;
   if (pairs) {
     KernelTimer timer(c, EBK_FFN_GATEUP_PAIR, st);
-    e = launch_ffn<1, true>(c, st, tm_x, tm_xs, c->tm_gate, c->tm_up, c->work1p, c->act, g.I, g.I, g.H, tm_xl);
+    e = launch_swap<1>(c, st, tok_x, c->tm_gate, c->tm_up, c->work1p, c->act, g.I, g.I, g.H);
   }
   if (e == cudaSuccess) {
     KernelTimer timer(c, EBK_FFN_GATEUP, st);
-    e = launch_ffn<1, false>(c, st, tm_x, tm_xs, c->tm_gate, c->tm_up, c->work1, c->act, g.I, g.I, g.H, tm_xl);
+    e = launch_ffn<1>(c, st, tm_x, tm_xs, c->tm_gate, c->tm_up, c->work1, c->act, g.I, g.I, g.H, tm_xl);
   }
   if (e == cudaSuccess && pairs) {
     KernelTimer timer(c, EBK_FFN_DOWN_PAIR, st);
-    e = launch_ffn<2, true>(c, st, tm_a, tm_as, c->tm_down_half, c->tm_down_half, c->work2p, (bf16*)yp, g.H, g.H, g.I, tm_al);
+    e = launch_swap<2>(c, st, tok_a, c->tm_down_half, c->tm_down_half, c->work2p, (bf16*)yp, g.H, g.H, g.I);
   }
   if (e == cudaSuccess) {
     KernelTimer timer(c, EBK_FFN_DOWN, st);
-    e = launch_ffn<2, false>(c, st, tm_a, tm_as, c->tm_down, c->tm_down, c->work2, (bf16*)yp, g.H, g.H, g.I, tm_al);
+    e = launch_ffn<2>(c, st, tm_a, tm_as, c->tm_down, c->tm_down, c->work2, (bf16*)yp, g.H, g.H, g.I, tm_al);
   }
   if (e != cudaSuccess) return ebi_check_cuda(c, e, "expert_ffn launch");
   EB_LAUNCH_CHECK(c, "expert_ffn");

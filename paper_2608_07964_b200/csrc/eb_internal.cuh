@@ -80,8 +80,9 @@ struct eb_ctx {
   int32_t* chunk_base = nullptr;   // [max_chunks][E]
   int32_t* group_size = nullptr;   // [G_cap]
   int32_t* mtile_pref = nullptr;   // [G_cap + 1] 128-row tiles before each group
-  int32_t* ptile_pref = nullptr;   // [G_cap + 1] 256-row pair tiles before each group
+  int32_t* ptile_pref = nullptr;   // [G_cap + 1] pair tiles before each entry of ppgroup
   int32_t* pgroup = nullptr;       // [G_cap] group at each position of the processing order
+  int32_t* ppgroup = nullptr;      // [G_cap] pair groups (more than 128 rows) in the order their tiles are listed
   int32_t* pchunks = nullptr;      // [G_cap] 32-row chunks of a merged shared-expert class, -1 otherwise
   int32_t* work_count = nullptr;   // [16]: tile counts of the four lists, group range, layers, device filter
   int4* work1 = nullptr;           // gate/up tile list
