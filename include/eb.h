@@ -63,7 +63,10 @@ enum { EB_MAX_MB = 16, EB_MAX_D = 16, EB_MAX_E = 256, EB_MAX_K = 8, EB_MAX_S = 8
 
 /* Length of the int32 `step_meta` array written by eb_permute:
  *   [0] R = rows of this step, [1] G = groups, [2] number of active layers,
- *   [3 .. 3+D] first group of every virtual device (D+1 entries), rest unused. */
+ *   [3 .. 3+D] first group of every virtual device (D+1 entries),
+ *   [EB_META_LEN-1] routing indices outside [0, E) met in topk_idx: each is skipped (its slot gets
+ *   pos = -1 and no row, it is never used as an index) and counted here; always 0 for indices
+ *   written by eb_route.  The entries in between are unused. */
 enum { EB_META_LEN = 32 };
 
 typedef struct {
@@ -250,8 +253,13 @@ enum { EB_NOALLOC_MAX_TOKENS = 4096 };
  * - The first call on each device resolves the array's device address (cudaGetSymbolAddress, with
  *   that device current); make that first call outside any stream capture.
  * - All calls on a device share the one array, which keeps the previous call's contents; the call
- *   re-initialises what it reads (tables copied, counters cleared) on `stream`.  Two calls whose
- *   work overlaps on the GPU (different streams, or different threads) race on it: serialise them.
+ *   re-initialises what it reads on `stream` (a set-up kernel rewrites the expert tables, which it
+ *   receives by value, and clears the counters; no host memory is read after the call returns).
+ *   Two calls whose work overlaps on the GPU (different streams, or different threads) race on the
+ *   array: serialise them.
+ * - The call works on whichever device is current, each device with its own copy of the array.
+ * - topk_idx and d_res are the caller's data here, not checked by a context: routing indices
+ *   outside [0, E) are skipped and counted in step_meta[EB_META_LEN-1], never dereferenced.
  * - `err` (host, may be NULL) receives a description of a failure, truncated to err_cap bytes. */
 eb_status eb_permute_noalloc(const eb_config* cfg, void* stream, const eb_batch* batch,
                              const eb_sched_result* d_res, const void* x, const int32_t* topk_idx,

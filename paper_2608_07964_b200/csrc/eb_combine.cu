@@ -47,7 +47,7 @@ combine_kernel(int n_tok, int H, int K, int team, const uint4* __restrict__ yp, 
   for (int v = threadIdx.x % team; v < vec; v += team) {
     uint4 r[KS];
 #pragma unroll
-    for (int s = 0; s < KS; ++s) r[s] = __ldg(yp + (size_t)p[s] * vec + v);
+    for (int s = 0; s < KS; ++s) r[s] = p[s] >= 0 ? __ldg(yp + (size_t)p[s] * vec + v) : make_uint4(0, 0, 0, 0);   // no row: adds 0
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int s = 0; s < KS; ++s) fma8(acc, r[s], w[s]);

@@ -98,7 +98,10 @@ hist_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ 
   if ((run >> j) & 1u) {
     int t0 = bp.tok_off[j] + (c - bp.chunk_off[j]) * 32;
     int nt = min(32, bp.tok_off[j + 1] - t0);
-    for (int a = lane; a < nt * K; a += 32) atomicAdd(&h[topk_idx[(size_t)t0 * K + a]], 1);
+    for (int a = lane; a < nt * K; a += 32) {
+      const int e = topk_idx[(size_t)t0 * K + a];
+      if ((unsigned)e < (unsigned)E) atomicAdd(&h[e], 1);   // an index outside [0, E) is skipped here and reported by rank
+    }
   }
   __syncwarp();
   for (int e = lane; e < E; e += 32) chunk_hist[(size_t)c * E + e] = h[e];
@@ -228,7 +231,8 @@ scan_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ 
 __global__ void __launch_bounds__(kWarps * 32)
 rank_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ res,
             const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ chunk_base,
-            const int32_t* __restrict__ group_off, int32_t* __restrict__ pos, int32_t* __restrict__ row_src) {
+            const int32_t* __restrict__ group_off, int32_t* __restrict__ pos, int32_t* __restrict__ row_src,
+            int32_t* __restrict__ step_meta) {
   EB_GRID_DEP_SYNC();
   __shared__ int s_next[kWarps][EB_MAX_E];
   __shared__ int s_dev_off[EB_MAX_D + 1];
@@ -259,6 +263,14 @@ rank_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __restrict__ 
     int a = a0 + lane;
     bool valid = a < nt * K;
     int e = valid ? topk_idx[(size_t)t0 * K + a] : -1 - lane;  // distinct dummies never match
+    if (valid && (unsigned)e >= (unsigned)E) {
+      // routing index outside [0, E) (only possible with tables not written by eb_route): never used as an
+      // index; the slot gets no row and the step's meta data counts it
+      pos[(size_t)(t0 + a / K) * KS + a % K] = -1;
+      atomicAdd(&step_meta[EB_META_LEN - 1], 1);
+      valid = false;
+      e = -1 - lane;
+    }
     unsigned peers = __match_any_sync(0xffffffffu, e);
     int before = __popc(peers & ((1u << lane) - 1u));
     int p = 0;
@@ -345,7 +357,10 @@ permute_fused_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __re
     if ((run >> j) & 1u) {
       const int t0 = bp.tok_off[j] + (c - bp.chunk_off[j]) * 32;
       const int nt = min(32, bp.tok_off[j + 1] - t0);
-      for (int a = lane; a < nt * K; a += 32) atomicAdd(&h[s_topk[t0 * K + a]], 1);
+      for (int a = lane; a < nt * K; a += 32) {
+        const int e = s_topk[t0 * K + a];
+        if ((unsigned)e < (unsigned)E) atomicAdd(&h[e], 1);
+      }
     }
   }
   __syncthreads();
@@ -443,8 +458,14 @@ permute_fused_kernel(ModelParams mp, BatchParams bp, const eb_sched_result* __re
     __syncwarp();
     for (int a0 = 0; a0 < nt * K; a0 += 32) {
       const int a = a0 + lane;
-      const bool valid = a < nt * K;
-      const int e = valid ? s_topk[t0 * K + a] : -1 - lane;
+      bool valid = a < nt * K;
+      int e = valid ? s_topk[t0 * K + a] : -1 - lane;
+      if (valid && (unsigned)e >= (unsigned)E) {   // as in rank_kernel: skipped and counted, never used as an index
+        pos[(size_t)(t0 + a / K) * KS + a % K] = -1;
+        atomicAdd(&step_meta[EB_META_LEN - 1], 1);
+        valid = false;
+        e = -1 - lane;
+      }
       const unsigned peers = __match_any_sync(0xffffffffu, e);
       const int before = __popc(peers & ((1u << lane) - 1u));
       if (valid) {
@@ -496,7 +517,7 @@ gather_kernel(int n_tok, int H, int KS, int team, const uint4* __restrict__ x, c
     if (v < vec) r = __ldg(src + v);
     for (int s = 0; s < KS; ++s) {
       const int p = __shfl_sync(0xffffffffu, my_pos, s);
-      if (v < vec) xp[(size_t)p * vec + v] = r;
+      if (v < vec && p >= 0) xp[(size_t)p * vec + v] = r;
     }
   }
 }
@@ -560,7 +581,7 @@ extern "C" eb_status eb_permute(eb_ctx* c, void* stream, const eb_batch* batch, 
     if (bp.n_chunks > 0) {
       KernelTimer timer(c, EBK_PERMUTE_RANK, st);
       ebi_launch(rank_kernel, dim3(chunk_blocks), dim3(kWarps * 32), 0, st, c->mp, bp, d_res, topk_idx,
-                 (const int32_t*)c->chunk_base, (const int32_t*)group_off, pos, row_src);
+                 (const int32_t*)c->chunk_base, (const int32_t*)group_off, pos, row_src, step_meta);
     }
   }
   if (bp.n_tok > 0) {
@@ -690,6 +711,25 @@ static __device__ __align__(256) int32_t g_noalloc_scratch[kNaWords];
 constexpr int kNaMaxDevices = 64;
 int32_t* g_noalloc_ptr[kNaMaxDevices] = {};
 
+// Expert tables of one call, handed to the set-up kernel by value (they travel in the launch's parameter
+// buffer, so no host memory has to outlive the call).
+struct NaTables {
+  int32_t n;
+  int32_t v[3 * EB_MAX_E + EB_MAX_D + 1];
+};
+static_assert(sizeof(NaTables) <= 4000, "kernel parameter space");
+
+// Writes the expert tables and clears the counters of the shared scratch array: every call starts from
+// the same state whatever the previous call left behind.
+__global__ void __launch_bounds__(256)
+noalloc_setup_kernel(const __grid_constant__ NaTables t, int32_t* __restrict__ d_tab, int32_t* __restrict__ d_hist, int n_hist,
+                     int32_t* __restrict__ d_gsize, int n_gsize) {
+  const int tid = blockIdx.x * blockDim.x + threadIdx.x, nthr = gridDim.x * blockDim.x;
+  for (int i = tid; i < t.n; i += nthr) d_tab[i] = t.v[i];
+  for (int i = tid; i < n_hist; i += nthr) d_hist[i] = 0;
+  for (int i = tid; i < n_gsize; i += nthr) d_gsize[i] = 0;
+}
+
 eb_status noalloc_fail(char* err, size_t cap, eb_status s, const char* msg) {
   if (err && cap) {
     size_t n = strlen(msg) < cap - 1 ? strlen(msg) : cap - 1;
@@ -719,9 +759,13 @@ extern "C" eb_status eb_permute_noalloc(const eb_config* cfg, void* stream, cons
     return noalloc_fail(err, err_cap, EB_ERR_UNSUPPORTED,
                         "eb_permute_noalloc handles at most EB_NOALLOC_MAX_TOKENS (4096) packed tokens: "
                         "its scratch is a fixed device array; use eb_permute with a workspace for more");
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNaMaxDevices)
+    return noalloc_fail(err, err_cap, EB_ERR_CUDA, "cudaGetDevice failed or device index too large");
   eb_ctx tmp;  // host-only helper for the shared argument checks; owns no device memory
   tmp.cfg = g;
   tmp.cfg.max_tokens = kNaMaxTokens;
+  tmp.device = dev;   // the checks compare against the current device: this call belongs to whichever device is current
   BatchParams bp;
   eb_status s = ebi_make_batch(&tmp, batch, &bp);
   if (s != EB_OK) return noalloc_fail(err, err_cap, s, tmp.err.c_str());
@@ -731,9 +775,6 @@ extern "C" eb_status eb_permute_noalloc(const eb_config* cfg, void* stream, cons
     return noalloc_fail(err, err_cap, EB_ERR_INVALID_ARG, "x / xp must be 16-byte aligned");
 
   // one-time set-up per device: resolve the device address of the scratch array
-  int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNaMaxDevices)
-    return noalloc_fail(err, err_cap, EB_ERR_CUDA, "cudaGetDevice failed or device index too large");
   if (!g_noalloc_ptr[dev]) {
     int32_t* p = nullptr;
     cudaError_t e = cudaGetSymbolAddress((void**)&p, g_noalloc_scratch);
@@ -747,7 +788,9 @@ extern "C" eb_status eb_permute_noalloc(const eb_config* cfg, void* stream, cons
   int32_t* d_gsize = d_cbase + kNaHistWords;
 
   // expert tables, same layout as a context's: e2d | dev_off | dev_list | e_local
-  int32_t tab[kNaTableWords];
+  NaTables tables;
+  int32_t* tab = tables.v;
+  tables.n = 3 * g.E + g.D + 1;
   int32_t* h_off = tab + g.E;
   int32_t* h_list = h_off + g.D + 1;
   int32_t* h_local = h_list + g.E;
@@ -771,10 +814,9 @@ extern "C" eb_status eb_permute_noalloc(const eb_config* cfg, void* stream, cons
   mp.e_local = mp.dev_list + g.E;
 
   cudaStream_t st = (cudaStream_t)stream;
-  cudaError_t ce = cudaMemcpyAsync(d_tab, tab, sizeof(int32_t) * (3 * g.E + g.D + 1), cudaMemcpyHostToDevice, st);
-  // the array keeps the previous call's contents: counters start from zero every call
-  if (ce == cudaSuccess) ce = cudaMemsetAsync(d_hist, 0, sizeof(int32_t) * (size_t)kNaHistWords, st);
-  if (ce == cudaSuccess) ce = cudaMemsetAsync(d_gsize, 0, sizeof(int32_t) * (size_t)kNaGroupWords, st);
+  // the array keeps the previous call's contents: tables rewritten, counters start from zero every call
+  noalloc_setup_kernel<<<64, 256, 0, st>>>(tables, d_tab, d_hist, kNaHistWords, d_gsize, kNaGroupWords);
+  cudaError_t ce = cudaGetLastError();
   if (ce != cudaSuccess) return noalloc_fail(err, err_cap, EB_ERR_CUDA, cudaGetErrorString(ce));
 
   const int gcap = EB_MAX_MB * (g.E + g.D * g.S);
@@ -783,7 +825,7 @@ extern "C" eb_status eb_permute_noalloc(const eb_config* cfg, void* stream, cons
   sizes_kernel<<<(gcap + kWarps - 1) / kWarps, kWarps * 32, 0, st>>>(mp, bp, d_res, d_hist, d_cbase, d_gsize);
   scan_kernel<<<1, 1024, 0, st>>>(mp, bp, d_res, d_gsize, group_off, group_w, step_meta);
   if (bp.n_chunks > 0)
-    rank_kernel<<<chunk_blocks, kWarps * 32, 0, st>>>(mp, bp, d_res, topk_idx, d_cbase, group_off, pos, row_src);
+    rank_kernel<<<chunk_blocks, kWarps * 32, 0, st>>>(mp, bp, d_res, topk_idx, d_cbase, group_off, pos, row_src, step_meta);
   if (bp.n_tok > 0) {
     const int team = team_for(g.H / 8), tpb = kGatherThreads / team;
     gather_kernel<<<(bp.n_tok + tpb - 1) / tpb, kGatherThreads, 0, st>>>(bp.n_tok, g.H, g.K + g.S, team, (const uint4*)x,
