@@ -78,26 +78,21 @@ static size_t carve(eb_ctx* c, char* base) {
   };
   c->max_chunks = (g.max_tokens + 31) / 32 + EB_MAX_MB;
   int rows = ebi_rows_cap(c), gcap = ebi_groups_cap(c);
-  c->max_mtiles = rows / 128 + gcap;
-  c->max_work1 = c->max_mtiles * ((g.I + 127) / 128);
-  c->max_work2 = c->max_mtiles * ((g.H + 255) / 256);
-  const int max_ptiles = rows / 256 + gcap;
-  c->max_work1p = max_ptiles * ((g.I + 255) / 256);   // pair tiles: 256 outputs (gate/up), 512 outputs (down)
-  c->max_work2p = max_ptiles * ((g.H + 511) / 512);
+  c->max_tiles = rows / 256 + gcap;                    // a group of r rows has ceil(r / 256) tiles
+  c->max_work1 = c->max_tiles * ((g.I + 255) / 256);   // 256 outputs per gate/up tile
+  c->max_work2 = c->max_tiles * ((g.H + 511) / 512);   // 512 outputs per down tile
   c->chunk_hist = (int32_t*)take(sizeof(int32_t) * (size_t)c->max_chunks * g.E);
   c->chunk_base = (int32_t*)take(sizeof(int32_t) * (size_t)c->max_chunks * g.E);
   c->group_size = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
-  c->mtile_pref = (int32_t*)take(sizeof(int32_t) * (size_t)(gcap + 1));
-  c->ptile_pref = (int32_t*)take(sizeof(int32_t) * (size_t)(gcap + 1));
   c->pgroup = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
-  c->ppgroup = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
-  c->pchunks = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
+  c->pslots = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
+  c->pcost = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
+  c->order = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
+  c->tile_pref = (int32_t*)take(sizeof(int32_t) * (size_t)(gcap + 1));
   c->work_count = (int32_t*)take(sizeof(int32_t) * 16);
   c->work1 = (int4*)take(sizeof(int4) * (size_t)c->max_work1);
   c->work2 = (int4*)take(sizeof(int4) * (size_t)c->max_work2);
-  c->work1p = (int4*)take(sizeof(int4) * (size_t)c->max_work1p);
-  c->work2p = (int4*)take(sizeof(int4) * (size_t)c->max_work2p);
-  c->slots = (int2*)take(sizeof(int2) * 8 * (size_t)c->max_mtiles);
+  c->slots = (int2*)take(sizeof(int2) * 16 * (size_t)c->max_tiles);
   c->act = (bf16*)take(sizeof(bf16) * (size_t)rows * g.I);
   return off;
 }
@@ -351,7 +346,7 @@ extern "C" eb_status eb_selftest_bounded_wait(eb_ctx* c, void* stream, int64_t l
 
 static const char* kKernelNames[EBK_COUNT] = {
     "route", "schedule", "permute_hist", "permute_sizes", "permute_scan", "permute_rank",
-    "permute_gather", "ffn_plan", "ffn_fill", "ffn_gateup", "ffn_down", "ffn_gateup_pair", "ffn_down_pair", "combine", "permute_fused"};
+    "permute_gather", "ffn_plan", "ffn_fill", "ffn_gateup", "ffn_down", "combine", "permute_fused"};
 
 extern "C" int32_t eb_num_kernels(void) { return EBK_COUNT; }
 extern "C" const char* eb_kernel_name(int32_t i) { return (i >= 0 && i < EBK_COUNT) ? kKernelNames[i] : ""; }

@@ -27,8 +27,6 @@ enum EbKernel {
   EBK_FFN_FILL,
   EBK_FFN_GATEUP,
   EBK_FFN_DOWN,
-  EBK_FFN_GATEUP_PAIR,
-  EBK_FFN_DOWN_PAIR,
   EBK_COMBINE,
   EBK_PERMUTE_FUSED,
   EBK_COUNT
@@ -66,12 +64,8 @@ struct eb_ctx {
   const bf16* w_gate = nullptr;
   const bf16* w_up = nullptr;
   const bf16* w_down = nullptr;
-  CUtensorMap tm_gate, tm_up, tm_down, tm_down_half;
-  int pair_grid = 0;               // CTAs launched for the CTA-pair kernels (0: pairs unavailable)
-  // Host-side hint left by the last eb_permute: the largest number of tokens sitting at one layer,
-  // an upper bound on the rows of any group of that step, and the step_meta buffer it belongs to.
-  int32_t hint_max_group_rows = -1;
-  const int32_t* hint_meta = nullptr;
+  CUtensorMap tm_gate, tm_up, tm_down;
+  int pair_grid = 0;               // CTAs launched for the expert kernels: two per 2-CTA cluster the device holds at once
 
   // workspace carve-up
   void* ws = nullptr;
@@ -79,19 +73,17 @@ struct eb_ctx {
   int32_t* chunk_hist = nullptr;   // [max_chunks][E]
   int32_t* chunk_base = nullptr;   // [max_chunks][E]
   int32_t* group_size = nullptr;   // [G_cap]
-  int32_t* mtile_pref = nullptr;   // [G_cap + 1] 128-row tiles before each group
-  int32_t* ptile_pref = nullptr;   // [G_cap + 1] pair tiles before each entry of ppgroup
   int32_t* pgroup = nullptr;       // [G_cap] group at each position of the processing order
-  int32_t* ppgroup = nullptr;      // [G_cap] pair groups (more than 128 rows) in the order their tiles are listed
-  int32_t* pchunks = nullptr;      // [G_cap] 32-row chunks of a merged shared-expert class, -1 otherwise
-  int32_t* work_count = nullptr;   // [16]: tile counts of the four lists, group range, layers, device filter
+  int32_t* pslots = nullptr;       // [G_cap] 16-row slots of the merged shared-expert class of the position, -1 otherwise
+  int32_t* pcost = nullptr;        // [G_cap] tiles | columns << 20 of the position
+  int32_t* order = nullptr;        // [G_cap] positions that own tiles, widest tiles first
+  int32_t* tile_pref = nullptr;    // [G_cap + 1] tiles before each entry of `order`
+  int32_t* work_count = nullptr;   // [16]: tile counts of the two lists, group range, layers, device filter
   int4* work1 = nullptr;           // gate/up tile list
   int4* work2 = nullptr;           // down tile list
-  int4* work1p = nullptr;          // gate/up tile list of the CTA-pair kernel
-  int4* work2p = nullptr;          // down tile list of the CTA-pair kernel
-  int2* slots = nullptr;           // [8 * max_mtiles] (first row, rows) of the 16-row slots of merged tiles
+  int2* slots = nullptr;           // [16 * max_tiles] (first row, rows) of the 16-row slots of merged tiles
   bf16* act = nullptr;             // [R_cap][I]
-  int32_t max_chunks = 0, max_mtiles = 0, max_work1 = 0, max_work2 = 0, max_work1p = 0, max_work2p = 0;
+  int32_t max_chunks = 0, max_tiles = 0, max_work1 = 0, max_work2 = 0;
 
   bool fused_attr_set = false;
   // eb_step_host_submit / eb_step_host_wait: copy streams and per-slot events, created on first use

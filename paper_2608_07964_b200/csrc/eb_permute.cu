@@ -538,19 +538,6 @@ extern "C" eb_status eb_permute(eb_ctx* c, void* stream, const eb_batch* batch, 
   if (!ebi_aligned16(x) || !ebi_aligned16(xp)) return ebi_fail(c, EB_ERR_INVALID_ARG, "x / xp must be 16-byte aligned");
   if (!c->ws) return ebi_fail(c, EB_ERR_WORKSPACE, "no workspace set");
   cudaStream_t st = (cudaStream_t)stream;
-  {
-    // upper bound on the rows of any group: tokens of pool members sharing a layer (performance hint
-    // for the expert pass; correctness never depends on it)
-    int best = 0;
-    for (int j = 0; j < bp.n_mb; ++j) {
-      int tot = 0;
-      for (int j2 = 0; j2 < bp.n_mb; ++j2)
-        if (bp.layer[j2] == bp.layer[j] && ((batch->pool_mask >> j2) & 1u)) tot += bp.tok_off[j2 + 1] - bp.tok_off[j2];
-      best = tot > best ? tot : best;
-    }
-    c->hint_max_group_rows = best;
-    c->hint_meta = step_meta;
-  }
   const int gcap = ebi_groups_cap(c);
   const int chunk_blocks = (bp.n_chunks + kWarps - 1) / kWarps;
   if (bp.n_chunks <= kFusedMaxChunks && gcap <= kFusedMaxGroups) {

@@ -38,7 +38,7 @@ def test_host_side_argument_errors_need_no_gpu():
     lib = binding.load_library()
     assert lib.eb_status_string(0) == b"ok"
     assert lib.eb_status_string(5) == b"device-side wait timed out"
-    assert lib.eb_num_kernels() == 15
+    assert lib.eb_num_kernels() == 13
     assert lib.eb_kernel_name(9) == b"ffn_gateup"
     h = ctypes.c_void_p()
     e2d = (ctypes.c_int32 * 4)(0, 0, 1, 1)
