@@ -2,9 +2,10 @@
 """Benchmark of one cross-layer MoE step (route -> schedule -> permute -> grouped expert FFN ->
 combine) on seeded synthetic inputs shaped like the benchmark configurations.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4] [--impl ours|reference]
 
-Prints ONE JSON line.  `value` is tokens of the chosen micro-batches per second with all inputs
+Prints ONE JSON line.  The default workload is the large-expert shape (the largest single-GPU configuration);
+the decode, fine-grained and layer-0 shapes are reported compactly under detail.other_workloads.  `value` is tokens of the chosen micro-batches per second with all inputs
 resident in HBM; `e2e` is the same with pinned host buffers, every step copying its inputs in and its result
 out inside the timed region, two steps in flight (eb_step_host_submit / eb_step_host_wait;
 `e2e.one_step_at_a_time` is the blocking eb_step_host).  With N > 1 (torchrun) every rank runs an independent replica
@@ -33,16 +34,14 @@ from paper_2608_07964_b200 import synth  # noqa: E402
 
 METRIC = "cross-layer MoE step tokens/s"
 UNIT = "tokens/s"
-# Kernels per step: route 2, schedule 1, permute 5, expert pass 4 or 6 (plan, fill, gate/up and down on single
-# CTAs, plus their CTA-pair launches when a group can exceed 128 rows), combine 1.  bench counts them from the
-# library's own launch counter.
+# Kernels per step: route, schedule, permute (one fused kernel or four, plus the gather), expert pass 4 (plan, fill,
+# gate/up, down), combine 1.  bench counts them from the library's own launch counter.
 
-# DRAM traffic of the dominant kernel (ffn gate/up) from an ncu capture: dram__bytes_read.sum +
-# dram__bytes_write.sum over the algorithmic bytes of the captured launch.  The capture ran on the
-# 6-layer cut of the decode shape (profiles/ffn_c2small_ncu_full.md); traffic grows in proportion to
-# the weight bytes streamed, so a full launch is that ratio times its own algorithmic bytes.
-NCU_TRAFFIC_RATIO = {"c2": (1.488622e9 + 7.138816e6) / 1487011840.0,
-                     "c2small": (1.488622e9 + 7.138816e6) / 1487011840.0}
+# DRAM traffic of the dominant kernel (ffn gate/up) from an ncu capture: (dram__bytes_read.sum +
+# dram__bytes_write.sum) over the algorithmic bytes of the captured launch.  The captures ran on cut-down cases
+# of the same shapes (a full-size capture would hold tens of GB); traffic grows in proportion to the weight
+# bytes streamed, so a full launch is that ratio times its own algorithmic bytes.
+NCU_TRAFFIC_RATIO = {}
 
 
 def measured_peaks():
@@ -68,7 +67,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._pump, daemon=True).start()
         except Exception:
@@ -257,25 +256,25 @@ def workload_config(wl):
 
 
 # ----------------------------------------------------------------------------------------------
-def run_ours(args, wl):
-    from paper_2608_07964_b200 import binding as B
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    dist = None
-    local = local % max(1, torch.cuda.device_count())
-    if world > 1:
-        import torch.distributed as dist
-        if args.dist_backend == "nccl":
-            dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
-        else:
-            dist.init_process_group(args.dist_backend)
-    torch.cuda.set_device(local)
-    device = f"cuda:{local}"
-    red_device = device if args.dist_backend == "nccl" else "cpu"   # where the timing reductions live
-    wl = replica_workload(wl, rank)
-    peaks = measured_peaks()
+def roof_of(nbytes, flops, ms, peaks):
+    """Roofline entry of one launch: the bound is whichever of bytes / HBM bandwidth and flops / tensor peak
+    takes longer with the measured peaks; achieved and frac are in that bound's unit."""
+    t = ms / 1e3
+    if nbytes / (peaks["hbm"] * 1e9) >= flops / (peaks["tensor"] * 1e12):
+        ach = nbytes / t / 1e9
+        d = dict(bound="hbm", achieved=ach, peak=peaks["hbm"], unit="GB/s", frac=ach / peaks["hbm"])
+    else:
+        ach = flops / t / 1e12
+        d = dict(bound="tensor", achieved=ach, peak=peaks["tensor"], unit="TFLOP/s", frac=ach / peaks["tensor"])
+    d.update(ms=ms, algorithmic_bytes=nbytes, algorithmic_flops=flops, peak_source=peaks["src"])
+    return d
 
+
+def measure(args, wl, device, local, dist, full):
+    """One workload on this rank: device-resident step time, per-kernel times, rooflines, idle block; with
+    `full` also the clock samples, the end-to-end figure and the CPU baseline.  Frees its device memory."""
+    from paper_2608_07964_b200 import binding as B
+    peaks = measured_peaks()
     step = B.from_workload(wl, device=device)
     wg, wu, wd = (synth.all_weights(wl, k, device) for k in ("gate", "up", "down"))
     step.bind_weights(wg, wu, wd)
@@ -286,6 +285,7 @@ def run_ours(args, wl):
     batch = B.Batch(wl.tok_off, wl.layers)
     m = wl.m
     run = lambda: step.eb_step(batch, m)
+    captured = None
     if args.graph:
         run()
         torch.cuda.synchronize()
@@ -307,16 +307,17 @@ def run_ours(args, wl):
         run()
     barrier()
     sampler = ClockSampler(local)
-    sampler.start()
-    time.sleep(0.25)
+    if full:
+        sampler.start()
+        time.sleep(0.25)
     t0 = time.time()
     launches0 = B.launch_count()
     ms = timed(run, args.steps)
     launches = B.launch_count() - launches0
-    if args.graph:
+    if captured is not None:
         launches = captured * args.steps
     t1 = time.time()
-    clocks = sampler.stop(t0, t1)
+    clocks = sampler.stop(t0, t1) if full else None
     barrier()
     status = step.device_status()
     sched = step.sched_result()
@@ -332,107 +333,157 @@ def run_ours(args, wl):
     step.set_timing(False)
     kern_ms = {k: sum(v) / len(v) for k, v in per.items()}
 
+    res = dict(wl=wl, ms=ms, launches=launches, clocks=clocks, status=status, sched=sched, tokens_run=tokens_run,
+               kern_ms=kern_ms, ms_e2e=float("nan"), ms_e2e_blocking=float("nan"))
+
     # ---- end to end with host buffers
-    h_logits = logits.cpu().pin_memory()
-    h_x = x.cpu().pin_memory()
-    h_out = torch.empty((T, wl.H), dtype=torch.bfloat16).pin_memory()
-    run_host = lambda: step.eb_step_host(batch, m, h_logits, h_x, h_out)
-    side = torch.cuda.Stream()      # a stream of its own: the legacy default stream adds implicit synchronisation
-    side.wait_stream(torch.cuda.current_stream())
-    # the same with two steps in flight (eb_step_host_submit / eb_step_host_wait): the copies of one step overlap
-    # the kernels of the other; every step still copies its inputs in and its result out inside the timed region
-    depth = 2
-    h_outs = [torch.empty((T, wl.H), dtype=torch.bfloat16).pin_memory() for _ in range(depth)]
+    if full:
+        h_logits = logits.cpu().pin_memory()
+        h_x = x.cpu().pin_memory()
+        h_out = torch.empty((T, wl.H), dtype=torch.bfloat16).pin_memory()
+        run_host = lambda: step.eb_step_host(batch, m, h_logits, h_x, h_out)
+        side = torch.cuda.Stream()      # a stream of its own: the legacy default stream adds implicit synchronisation
+        side.wait_stream(torch.cuda.current_stream())
+        # the same with two steps in flight (eb_step_host_submit / eb_step_host_wait): the copies of one step overlap
+        # the kernels of the other; every step still copies its inputs in and its result out inside the timed region
+        depth = 2
+        h_outs = [torch.empty((T, wl.H), dtype=torch.bfloat16).pin_memory() for _ in range(depth)]
 
-    def run_pipelined(n):
-        for i in range(n):
-            s = i % depth
-            if i >= depth:
+        def run_pipelined(n):
+            for i in range(n):
+                s = i % depth
+                if i >= depth:
+                    step.step_host_wait(s)
+                step.step_host_submit(s, batch, m, h_logits, h_x, h_outs[s])
+            for s in range(min(depth, n)):
                 step.step_host_wait(s)
-            step.step_host_submit(s, batch, m, h_logits, h_x, h_outs[s])
-        for s in range(min(depth, n)):
-            step.step_host_wait(s)
 
-    with torch.cuda.stream(side):
-        for _ in range(max(args.warmup, 3)):
-            run_host()
+        with torch.cuda.stream(side):
+            for _ in range(max(args.warmup, 3)):
+                run_host()
+            barrier()
+            res["ms_e2e_blocking"] = timed(run_host, args.steps)
+            run_pipelined(max(args.warmup, 3))
+            barrier()
+            res["ms_e2e"] = timed(lambda: run_pipelined(args.steps), 1)
         barrier()
-        ms_e2e_blocking = timed(run_host, args.steps)
-        run_pipelined(max(args.warmup, 3))
-        barrier()
-        ms_e2e = timed(lambda: run_pipelined(args.steps), 1)
-    barrier()
-    for h in h_outs:      # rows of deferred micro-batches are not written by a step
-        for j in range(wl.N):
-            if (sched["run_mask"] >> j) & 1:
-                a, b = wl.tok_off[j], wl.tok_off[j + 1]
-                assert torch.equal(h[a:b], h_out[a:b]), "pipelined host path disagrees with the blocking one"
+        for h in h_outs:      # rows of deferred micro-batches are not written by a step
+            for j in range(wl.N):
+                if (sched["run_mask"] >> j) & 1:
+                    a, b = wl.tok_off[j], wl.tok_off[j + 1]
+                    assert torch.equal(h[a:b], h_out[a:b]), "pipelined host path disagrees with the blocking one"
+
+    # ---- algorithmic work and rooflines of the two expert launches
+    meta = step.meta()
+    alg = algorithmic_bytes(wl, step.group_off.cpu().numpy(), step.group_w.cpu().numpy(), meta["groups"])
+    t_gu, t_dn = kern_ms.get("ffn_gateup", float("nan")), kern_ms.get("ffn_down", float("nan"))
+    roofs = dict(ffn_gateup=roof_of(alg["gateup"], alg["gateup_flops"], t_gu, peaks),
+                 ffn_down=roof_of(alg["down"], alg["down_flops"], t_dn, peaks))
+    ffn_flops = alg["gateup_flops"] + alg["down_flops"]
+    ffn_bytes = alg["gateup"] + alg["down"]
+    t_ffn = (t_gu + t_dn) / 1e3
+    move = 2 * (tokens_run * wl.H + alg["rows"] * wl.H)      # gather: read T_run rows, write R rows; combine the reverse
+    t_g, t_c = kern_ms.get("permute_gather", float("nan")) / 1e3, kern_ms.get("combine", float("nan")) / 1e3
+    res.update(alg=alg, roofs=roofs, extra=dict(
+        kernel_ms=kern_ms, launches=roofs,
+        ffn=dict(tflops=ffn_flops / t_ffn / 1e12, frac_tensor_peak=ffn_flops / t_ffn / 1e12 / peaks["tensor"],
+                 frac_tensor_sustained=ffn_flops / t_ffn / 1e12 / peaks["tensor_sustained"],
+                 gbs=ffn_bytes / t_ffn / 1e9, frac_hbm=ffn_bytes / t_ffn / 1e9 / peaks["hbm"],
+                 active_groups=alg["active_groups"], distinct_matrices=alg["distinct_matrices"], rows=alg["rows"]),
+        front_end_ms=sum(v for k, v in kern_ms.items() if not k.startswith("ffn_gate") and not k.startswith("ffn_down")),
+        permute_gather=dict(bytes=move, gbs=move / t_g / 1e9, frac_hbm=move / t_g / 1e9 / peaks["hbm"],
+                            frac_hbm_nominal_8tbs=move / t_g / 1e9 / 8000.0),
+        combine=dict(bytes=move, gbs=move / t_c / 1e9, frac_hbm=move / t_c / 1e9 / peaks["hbm"],
+                     frac_hbm_nominal_8tbs=move / t_c / 1e9 / 8000.0)))
+    res["idle"] = idle_report(step, batch, wl, sched, B) if dist is None and not args.no_idle else None
+
+    res["cpu"] = None
+    if full and dist is None and not args.no_cpu_baseline:
+        get = lazy_cpu_weights(wl, device)
+        lg, xx = logits.cpu().numpy(), x.float().cpu().numpy()
+        oracle_step_sample(wl, lg, xx, get, 4.0)          # stages the sampled weights on the host
+        r = oracle_step_sample(wl, lg, xx, get, 12.0)
+        res["cpu"] = dict(value=r["tokens"] / r["seconds"], unit=UNIT, cores=cpu_threads(), kind="oracle",
+                          sample=(f"oracle whole step; expert pass over the first {r['groups']} non-empty groups "
+                                  f"({r['rows']} of {r['rows_total']} rows), other stages scaled to that share; "
+                                  f"{r['seconds']:.1f} s of CPU work"),
+                          stage_seconds={k: round(v, 4) for k, v in r["stages"].items()})
+    step.close()
+    del wg, wu, wd, step
+    torch.cuda.empty_cache()
+    return res
+
+
+def compact(res, peaks):
+    """Sub-line of a secondary workload."""
+    wl, ex = res["wl"], res["extra"]
+    ms_step = res["ms"] / res["steps"]
+    g = ex["launches"]["ffn_gateup"]
+    return dict(workload=workload_config(wl)["workload"], ms_per_step=ms_step,
+                tokens_per_s=res["tokens_run"] / (ms_step / 1e3), device_status=res["status"],
+                gateup=dict(bound=g["bound"], frac=g["frac"], ms=g["ms"]),
+                down=dict(bound=ex["launches"]["ffn_down"]["bound"], frac=ex["launches"]["ffn_down"]["frac"],
+                          ms=ex["launches"]["ffn_down"]["ms"]),
+                expert_pass_tflops=ex["ffn"]["tflops"], expert_pass_frac_burst=ex["ffn"]["frac_tensor_peak"],
+                expert_pass_frac_sustained=ex["ffn"]["frac_tensor_sustained"], expert_pass_frac_hbm=ex["ffn"]["frac_hbm"],
+                front_end_ms=ex["front_end_ms"], gather_gbs=ex["permute_gather"]["gbs"], combine_gbs=ex["combine"]["gbs"],
+                idle=res["idle"])
+
+
+def run_ours(args, wl):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    local = local % max(1, torch.cuda.device_count())
+    if world > 1:
+        import torch.distributed as dist
+        if args.dist_backend == "nccl":
+            dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+        else:
+            dist.init_process_group(args.dist_backend)
+    torch.cuda.set_device(local)
+    device = f"cuda:{local}"
+    red_device = device if args.dist_backend == "nccl" else "cpu"   # where the timing reductions live
+    wl = replica_workload(wl, rank)
+    peaks = measured_peaks()
+
+    res = measure(args, wl, device, local, dist, full=True)
+    res["steps"] = args.steps
 
     # ---- reductions over ranks
-    ms_max, ms_e2e_max, tok_total = reduce_over_ranks(dist, red_device, ms, ms_e2e, float(tokens_run))
+    ms_max, ms_e2e_max, tok_total = reduce_over_ranks(dist, red_device, res["ms"], res["ms_e2e"], float(res["tokens_run"]))
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
-    meta = step.meta()
-    goff = step.group_off.cpu().numpy()
-    alg = algorithmic_bytes(wl, goff, step.group_w.cpu().numpy(), meta["groups"])
+    T = wl.T_tot
     ms_step = ms_max / args.steps
     value = tok_total / (ms_step / 1e3)
-    # dominant kernel: the gate/up pass of the grouped expert FFN
-    # a step's groups are split between the single-CTA and the CTA-pair launch of the same kernel
-    t_gu = (kern_ms.get("ffn_gateup", float("nan")) + kern_ms.get("ffn_gateup_pair", 0.0)) / 1e3
-    t_dn = (kern_ms.get("ffn_down", float("nan")) + kern_ms.get("ffn_down_pair", 0.0)) / 1e3
-    hbm_time = alg["gateup"] / (peaks["hbm"] * 1e9)
-    tensor_time = alg["gateup_flops"] / (peaks["tensor"] * 1e12)
-    if hbm_time >= tensor_time:
-        achieved = alg["gateup"] / t_gu / 1e9
-        roof = dict(bound="hbm", achieved=achieved, peak=peaks["hbm"], unit="GB/s", frac=achieved / peaks["hbm"])
-    else:
-        achieved = alg["gateup_flops"] / t_gu / 1e12
-        roof = dict(bound="tensor", achieved=achieved, peak=peaks["tensor"], unit="TFLOP/s", frac=achieved / peaks["tensor"])
-    roof.update(kernel="ffn_gateup", peak_source=peaks["src"], traffic=(NCU_TRAFFIC_RATIO[wl.name] * alg["gateup"] if wl.name in NCU_TRAFFIC_RATIO else None),
-                algorithmic_bytes=alg["gateup"], algorithmic_flops=alg["gateup_flops"], ms=t_gu * 1e3)
-    ffn_flops = alg["gateup_flops"] + alg["down_flops"]
-    ffn_bytes = alg["gateup"] + alg["down"]
-    t_ffn = t_gu + t_dn
-    move = 2 * (sum(wl.T for j in range(wl.N) if (sched["run_mask"] >> j) & 1) * wl.H + alg["rows"] * wl.H)
-    extra = dict(
-        kernel_ms=kern_ms,
-        ffn=dict(tflops=ffn_flops / t_ffn / 1e12, frac_tensor_peak=ffn_flops / t_ffn / 1e12 / peaks["tensor"],
-                 frac_tensor_sustained=ffn_flops / t_ffn / 1e12 / peaks["tensor_sustained"],
-                 gbs=ffn_bytes / t_ffn / 1e9, frac_hbm=ffn_bytes / t_ffn / 1e9 / peaks["hbm"],
-                 down_gbs=alg["down"] / t_dn / 1e9, active_groups=alg["active_groups"],
-                 distinct_matrices=alg["distinct_matrices"], rows=alg["rows"]),
-        permute_gather_gbs=move / (kern_ms.get("permute_gather", float("nan")) / 1e3) / 1e9,
-        combine_gbs=move / (kern_ms.get("combine", float("nan")) / 1e3) / 1e9,
-        permute_gather_frac_hbm=move / (kern_ms.get("permute_gather", float("nan")) / 1e3) / 1e9 / peaks["hbm"],
-        combine_frac_hbm=move / (kern_ms.get("combine", float("nan")) / 1e3) / 1e9 / peaks["hbm"],
-    )
-    idle = idle_report(step, batch, wl, sched, B) if world == 1 and not args.no_idle else None
-
-    cpu = None
-    if world == 1 and not args.no_cpu_baseline:
-        get = lazy_cpu_weights(wl, device)
-        lg, xx = logits.cpu().numpy(), x.float().cpu().numpy()
-        oracle_step_sample(wl, lg, xx, get, 4.0)          # stages the sampled weights on the host
-        r = oracle_step_sample(wl, lg, xx, get, 12.0)
-        cpu = dict(value=r["tokens"] / r["seconds"], unit=UNIT, cores=cpu_threads(), kind="oracle",
-                   sample=(f"oracle whole step; expert pass over the first {r['groups']} non-empty groups "
-                           f"({r['rows']} of {r['rows_total']} rows), other stages scaled to that share; "
-                           f"{r['seconds']:.1f} s of CPU work"))
+    # dominant kernel: the gate/up launch of the grouped expert FFN
+    roof = dict(res["roofs"]["ffn_gateup"])
+    roof.update(kernel="ffn_gateup",
+                traffic=(NCU_TRAFFIC_RATIO[wl.name] * roof["algorithmic_bytes"] if wl.name in NCU_TRAFFIC_RATIO else None))
+    extra = res["extra"]
+    if world == 1 and args.others:
+        extra["other_workloads"] = {}
+        for name in args.others.split(","):
+            sub = measure(args, named_workload(name), device, local, None, full=False)
+            sub["steps"] = args.steps
+            extra["other_workloads"][name] = compact(sub, peaks)
 
     h2d = T * wl.E * 4 + T * wl.H * 2
     d2h = T * wl.H * 2 + 96
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
-                data="synthetic", config=workload_config(wl), clocks=clocks,
+                data="synthetic", config=workload_config(wl), clocks=res["clocks"],
                 e2e=dict(value=tok_total / (ms_e2e_max / args.steps / 1e3), unit=UNIT, h2d_bytes_per_step=h2d,
                          d2h_bytes_per_step=d2h, mode="host buffers, 2 steps in flight (eb_step_host_submit/_wait)",
-                         one_step_at_a_time=tokens_run / (ms_e2e_blocking / args.steps / 1e3)),
-                gpu_launches=launches, roofline=roof, cpu_baseline=cpu,
-                tokens_per_step=tok_total, run_mask=sched["run_mask"], device_status=status, idle=idle, detail=extra)
+                         one_step_at_a_time=res["tokens_run"] / (res["ms_e2e_blocking"] / args.steps / 1e3)),
+                gpu_launches=res["launches"], roofline=roof, cpu_baseline=res["cpu"],
+                tokens_per_step=tok_total, run_mask=res["sched"]["run_mask"], device_status=res["status"],
+                idle=res["idle"], detail=extra)
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -468,10 +519,33 @@ def idle_report(step, batch, wl, sched, B):
         cap += D * max(tj)
     step.eb_step(batch, wl.m)
     torch.cuda.synchronize()
-    return dict(token_cross_layer=tok_cross, token_per_layer=tok_alone,
+    # what the emulated expert-parallel step costs is the slowest device's time: lead with that.  On shapes whose
+    # groups stream their weights (few rows per expert) a device's time follows the experts it touches, not its
+    # tokens, so the time-based idle fraction need not fall even though the slowest device gets faster.
+    return dict(step_max_ms_cross_layer=max(t_cross), sum_max_ms_per_layer=cap / D,
+                max_device_time_ratio=max(t_cross) / (cap / D) if cap else None,
+                token_cross_layer=tok_cross, token_per_layer=tok_alone,
                 time_cross_layer=1.0 - sum(t_cross) / (D * max(t_cross)),
                 time_per_layer=1.0 - busy / cap if cap else 0.0,
-                device_ms_cross_layer=t_cross, step_max_ms_cross_layer=max(t_cross), sum_max_ms_per_layer=cap / D)
+                device_ms_cross_layer=t_cross)
+
+
+def named_workload(name):
+    if name == "c3init":
+        # Algorithm 1's first step on the fine-grained shape: every micro-batch at layer 0 (tensor-bound groups)
+        wl = synth.workload("c3", layers_override=tuple([0] * 16))
+    elif name == "c3initsmall":
+        # c3init with the model cut to 2 layers (2.3 GB of weights): same kernels and tile shapes, small enough for ncu
+        wl = synth.workload("c3", L=2, layers_override=tuple([0] * 16))
+    elif name == "c4small":
+        # the large-expert shape cut to 2 layers and 2 micro-batches (5.6 GB of weights): small enough for ncu
+        wl = synth.workload("c4", L=2, N=2, m_override=2)
+    elif name == "c2small":
+        # the decode shape cut to 6 layers and 6 micro-batches (6.6 GB of weights): the case ncu captures run on
+        wl = synth.workload("c2", L=6, N=6)
+    else:
+        return synth.workload(name)
+    return synth.Workload(**{**wl.__dict__, "name": name})
 
 
 def main():
@@ -480,7 +554,11 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c2small", "c3", "c3init", "c3initsmall", "c4", "c4small"])
+    ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c2small", "c3", "c3init", "c3initsmall", "c4", "c4small"],
+                    help="the workload of the JSON line; c4 (large experts, 90 GB of weights) is the largest single-GPU one")
+    ap.add_argument("--others", default=None,
+                    help="comma-separated workloads reported compactly under detail.other_workloads "
+                         "(default: c2,c3,c3init when the main workload is c4; 'none' for none)")
     ap.add_argument("--graph", action="store_true", help="replay the step from a captured CUDA graph")
     ap.add_argument("--dist-backend", default="nccl", choices=["nccl", "gloo"],
                     help="process-group backend for the barrier and the timing reductions (replicas share no data)")
@@ -488,23 +566,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.workload == "c3init":
-        wl = synth.workload("c3", layers_override=tuple([0] * 16))
-        wl = synth.Workload(**{**wl.__dict__, "name": "c3init"})
-    elif args.workload == "c3initsmall":
-        # c3init with the model cut to 2 layers (2.3 GB of weights): same kernels and tile shapes, small enough for ncu
-        wl = synth.workload("c3", L=2, layers_override=tuple([0] * 16))
-        wl = synth.Workload(**{**wl.__dict__, "name": "c3initsmall"})
-    elif args.workload == "c4small":
-        # the large-expert shape cut to 2 layers and 2 micro-batches (5.6 GB of weights): small enough for ncu
-        wl = synth.workload("c4", L=2, N=2, m_override=2)
-        wl = synth.Workload(**{**wl.__dict__, "name": "c4small"})
-    elif args.workload == "c2small":
-        # the decode shape cut to 6 layers and 6 micro-batches (6.6 GB of weights): the case ncu captures run on
-        wl = synth.workload("c2", L=6, N=6)
-        wl = synth.Workload(**{**wl.__dict__, "name": "c2small"})
-    else:
-        wl = synth.workload(args.workload)
+    if args.others is None:
+        args.others = "c2,c3,c3init" if args.workload == "c4" else ""
+    if args.others == "none":
+        args.others = ""
+    wl = named_workload(args.workload)
     if args.impl == "reference":
         run_reference(args, wl)
     else:
