@@ -117,6 +117,7 @@ typedef struct {
   void* yp;
   int32_t* step_meta;
   void* out;
+  const void* residual; /* NULL: out = MoE output (eb_combine); else bf16 [max_tokens, H] added as in eb_combine_residual; may equal out */
 } eb_step_buffers;
 
 /* ---- life cycle ------------------------------------------------------------------------- */
@@ -201,9 +202,20 @@ eb_status eb_expert_ffn_device(eb_ctx* ctx, void* stream, const void* xp, const 
 eb_status eb_combine(eb_ctx* ctx, void* stream, const eb_batch* batch, const eb_sched_result* d_res,
                      const void* yp, const int32_t* pos, const float* topk_w, void* out);
 
+/* The same with the residual connection of the MoE block, Section 2.1: h_{l+1} = h'_l + MLP(h'_l).
+ * out[t] = (the sum of Eq. 1 above) + residual[t], the residual row added last in fp32, one rounding to
+ * bf16.  residual bf16 [T_tot, H] is the block's input h' (what eb_permute gathered from); it may be the
+ * same buffer as `out` (the hidden states are then updated in place; rows of micro-batches that did
+ * not run stay as they are).  residual == NULL is eb_combine. */
+eb_status eb_combine_residual(eb_ctx* ctx, void* stream, const eb_batch* batch, const eb_sched_result* d_res,
+                              const void* yp, const int32_t* pos, const float* topk_w, const void* residual,
+                              void* out);
+
 /* ---- whole step --------------------------------------------------------------------------- */
 
-/* The five calls back to back on `stream` with device-resident inputs (buf->logits, buf->x). */
+/* The five calls back to back on `stream` with device-resident inputs (buf->logits, buf->x); the
+ * aggregation adds buf->residual when it is not NULL (Algorithm 1's step for a model that carries its
+ * hidden states in buf->x: residual = out = x updates them in place). */
 eb_status eb_step(eb_ctx* ctx, void* stream, const eb_batch* batch, uint32_t route_mask, int32_t m,
                   eb_policy policy, const eb_step_buffers* buf);
 

@@ -40,12 +40,13 @@ class EbSchedResult(C.Structure):
 
 class EbStepBuffers(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("logits", "x", "topk_idx", "topk_w", "mb_load", "mb_cnt", "sched",
-                                          "group_off", "group_w", "row_src", "pos", "xp", "yp", "step_meta", "out")]
+                                          "group_off", "group_w", "row_src", "pos", "xp", "yp", "step_meta", "out",
+                                          "residual")]
 
 
 SYMBOLS = ["eb_create", "eb_destroy", "eb_bind_weights", "eb_workspace_bytes", "eb_set_workspace",
            "eb_rows_capacity", "eb_groups_capacity", "eb_route", "eb_schedule", "eb_permute",
-           "eb_expert_ffn_grouped", "eb_expert_ffn_device", "eb_combine", "eb_step", "eb_step_host",
+           "eb_expert_ffn_grouped", "eb_expert_ffn_device", "eb_combine", "eb_combine_residual", "eb_step", "eb_step_host",
            "eb_step_host_submit", "eb_step_host_wait",
            "eb_permute_noalloc", "eb_selftest_bounded_wait", "eb_check_permutation",
            "eb_device_status", "eb_num_kernels", "eb_kernel_name", "eb_set_timing", "eb_kernel_ms",
@@ -83,6 +84,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.eb_expert_ffn_device.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32]
     lib.eb_combine.argtypes = [vp, vp, C.POINTER(EbBatch), vp, vp, vp, vp, vp]
     lib.eb_step.argtypes = [vp, vp, C.POINTER(EbBatch), u32, i32, i32, C.POINTER(EbStepBuffers)]
+    lib.eb_combine_residual.argtypes = [vp, vp, C.POINTER(EbBatch), vp, vp, vp, vp, vp, vp]
     lib.eb_step_host.argtypes = [vp, vp, C.POINTER(EbBatch), u32, i32, i32, C.POINTER(EbStepBuffers), vp, vp, vp, vp]
     lib.eb_step_host_submit.argtypes = [vp, vp, C.POINTER(EbBatch), u32, i32, i32, C.POINTER(EbStepBuffers), vp, vp, vp, vp, i32]
     lib.eb_step_host_wait.argtypes = [vp, i32]
@@ -182,7 +184,11 @@ class MoEStep:
         self.out = mk((max_tokens, H), bf)
         self.bufs = EbStepBuffers(*[t.data_ptr() for t in (
             self.logits, self.x, self.topk_idx, self.topk_w, self.mb_load, self.mb_cnt, self.sched, self.group_off,
-            self.group_w, self.row_src, self.pos, self.xp, self.yp, self.step_meta, self.out)])
+            self.group_w, self.row_src, self.pos, self.xp, self.yp, self.step_meta, self.out)], None)
+        # the same buffers with the hidden states updated in place: out = x + MoE(x) (Section 2.1)
+        self.bufs_inplace = EbStepBuffers(*[t.data_ptr() for t in (
+            self.logits, self.x, self.topk_idx, self.topk_w, self.mb_load, self.mb_cnt, self.sched, self.group_off,
+            self.group_w, self.row_src, self.pos, self.xp, self.yp, self.step_meta, self.x)], self.x.data_ptr())
         self._weights = None
 
     # -- helpers -------------------------------------------------------------------------------
@@ -244,15 +250,26 @@ class MoEStep:
                                                       self.group_w.data_ptr(), self.step_meta.data_ptr(), self.yp.data_ptr(),
                                                       device))
 
-    def eb_combine(self, batch: Batch, out: Optional[torch.Tensor] = None):
+    def eb_combine(self, batch: Batch, out: Optional[torch.Tensor] = None, residual: Optional[torch.Tensor] = None,
+                   yp: Optional[torch.Tensor] = None):
         o = self.out if out is None else out
-        self._check(self.lib.eb_combine(self.ctx, _stream(), C.byref(batch.c), self.sched.data_ptr(), self.yp.data_ptr(),
-                                        self.pos.data_ptr(), self.topk_w.data_ptr(), o.data_ptr()))
+        y = self.yp if yp is None else yp
+        if residual is None:
+            self._check(self.lib.eb_combine(self.ctx, _stream(), C.byref(batch.c), self.sched.data_ptr(), y.data_ptr(),
+                                            self.pos.data_ptr(), self.topk_w.data_ptr(), o.data_ptr()))
+        else:
+            self._check(self.lib.eb_combine_residual(self.ctx, _stream(), C.byref(batch.c), self.sched.data_ptr(),
+                                                     y.data_ptr(), self.pos.data_ptr(), self.topk_w.data_ptr(),
+                                                     residual.data_ptr(), o.data_ptr()))
 
     # -- whole step ----------------------------------------------------------------------------
-    def eb_step(self, batch: Batch, m: int, policy: int = POLICY_MAXUTIL, route_mask: Optional[int] = None):
+    def eb_step(self, batch: Batch, m: int, policy: int = POLICY_MAXUTIL, route_mask: Optional[int] = None,
+                in_place: bool = False):
+        """The five calls back to back.  With `in_place` the hidden states self.x take x + MoE(x) for the chosen
+        micro-batches (the aggregation adds the residual and writes over x); otherwise the MoE output goes to self.out."""
         rm = ((1 << batch.n_mb) - 1) if route_mask is None else route_mask
-        self._check(self.lib.eb_step(self.ctx, _stream(), C.byref(batch.c), rm, m, policy, C.byref(self.bufs)))
+        bufs = self.bufs_inplace if in_place else self.bufs
+        self._check(self.lib.eb_step(self.ctx, _stream(), C.byref(batch.c), rm, m, policy, C.byref(bufs)))
 
     def eb_step_host(self, batch: Batch, m: int, h_logits: torch.Tensor, h_x: torch.Tensor, h_out: torch.Tensor,
                      policy: int = POLICY_MAXUTIL, route_mask: Optional[int] = None) -> Dict:
@@ -279,7 +296,7 @@ class MoEStep:
             out = mk((self.max_tokens, self.H), bf)
             bufs = EbStepBuffers(*[t.data_ptr() for t in (
                 logits, x, self.topk_idx, self.topk_w, self.mb_load, self.mb_cnt, sched, self.group_off,
-                self.group_w, self.row_src, self.pos, self.xp, self.yp, self.step_meta, out)])
+                self.group_w, self.row_src, self.pos, self.xp, self.yp, self.step_meta, out)], None)
             h_res = torch.zeros(C.sizeof(EbSchedResult), dtype=torch.uint8).pin_memory()   # pinned: the copy back is asynchronous
             self._slots[slot] = (bufs, h_res, (logits, x, sched, out))
         return self._slots[slot]

@@ -247,7 +247,8 @@ extern "C" eb_status eb_step(eb_ctx* c, void* stream, const eb_batch* batch, uin
   if ((s = eb_permute(c, stream, batch, b->sched, b->x, b->topk_idx, b->group_off, b->group_w, b->row_src, b->pos,
                       b->xp, b->step_meta)) != EB_OK) return s;
   if ((s = eb_expert_ffn_grouped(c, stream, b->xp, b->group_off, b->group_w, b->step_meta, b->yp)) != EB_OK) return s;
-  return eb_combine(c, stream, batch, b->sched, b->yp, b->pos, b->topk_w, b->out);
+  if (!ebi_aligned16(b->residual)) return ebi_fail(c, EB_ERR_INVALID_ARG, "residual not 16-byte aligned");
+  return eb_combine_residual(c, stream, batch, b->sched, b->yp, b->pos, b->topk_w, b->residual, b->out);
 }
 
 extern "C" eb_status eb_step_host(eb_ctx* c, void* stream, const eb_batch* batch, uint32_t route_mask, int32_t m,

@@ -1,4 +1,5 @@
-// eb_combine: weighted aggregation of Eq. 1 in gather form.
+// eb_combine: weighted aggregation of Eq. 1 in gather form; optionally the residual of the MoE block,
+// h_{l+1} = h'_l + MLP(h'_l) (Section 2.1), in the same pass.
 //
 // A team of threads per token, one 16-byte column vector each (a whole row in flight at once).  A
 // thread loads its vector from the K + S expert-output rows of the token (independent loads, all
@@ -27,7 +28,7 @@ __device__ __forceinline__ void fma8(float* acc, const uint4& v, float w) {
 template <int KS>
 __global__ void __launch_bounds__(kThreads)
 combine_kernel(int n_tok, int H, int K, int team, const uint4* __restrict__ yp, const int32_t* __restrict__ pos,
-               const float* __restrict__ topk_w, uint4* __restrict__ out) {
+               const float* __restrict__ topk_w, const uint4* residual, uint4* out) {   // residual may be `out` itself
   EB_GRID_DEP_SYNC();
   const int t = blockIdx.x * (kThreads / team) + threadIdx.x / team;   // team >= 32: a warp serves one token
   if (t >= n_tok) return;
@@ -48,9 +49,20 @@ combine_kernel(int n_tok, int H, int K, int team, const uint4* __restrict__ yp, 
     uint4 r[KS];
 #pragma unroll
     for (int s = 0; s < KS; ++s) r[s] = p[s] >= 0 ? __ldg(yp + (size_t)p[s] * vec + v) : make_uint4(0, 0, 0, 0);   // no row: adds 0
+    uint4 res = make_uint4(0, 0, 0, 0);
+    if (residual) res = residual[(size_t)t * vec + v];
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int s = 0; s < KS; ++s) fma8(acc, r[s], w[s]);
+    if (residual) {   // added last: out = sum + h'
+      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&res);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 f = __bfloat1622float2(h[i]);
+        acc[2 * i] += f.x;
+        acc[2 * i + 1] += f.y;
+      }
+    }
     uint4 o;
     __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&o);
 #pragma unroll
@@ -59,7 +71,7 @@ combine_kernel(int n_tok, int H, int K, int team, const uint4* __restrict__ yp, 
   }
 }
 
-typedef void (*combine_fn)(int, int, int, int, const uint4*, const int32_t*, const float*, uint4*);
+typedef void (*combine_fn)(int, int, int, int, const uint4*, const int32_t*, const float*, const uint4*, uint4*);
 
 // kernel for every slot count 1 .. kMaxSlots (entry 0 unused)
 template <int... Is>
@@ -72,12 +84,19 @@ const combine_fn* combine_table(std::integer_sequence<int, Is...>) {
 
 extern "C" eb_status eb_combine(eb_ctx* c, void* stream, const eb_batch* batch, const eb_sched_result* d_res,
                                 const void* yp, const int32_t* pos, const float* topk_w, void* out) {
+  return eb_combine_residual(c, stream, batch, d_res, yp, pos, topk_w, nullptr, out);
+}
+
+extern "C" eb_status eb_combine_residual(eb_ctx* c, void* stream, const eb_batch* batch, const eb_sched_result* d_res,
+                                         const void* yp, const int32_t* pos, const float* topk_w, const void* residual,
+                                         void* out) {
   if (!c) return EB_ERR_INVALID_ARG;
   BatchParams bp;
   eb_status s = ebi_make_batch(c, batch, &bp);
   if (s != EB_OK) return s;
   if (!d_res || !yp || !pos || !topk_w || !out) return ebi_fail(c, EB_ERR_INVALID_ARG, "null pointer");
-  if (!ebi_aligned16(yp) || !ebi_aligned16(out)) return ebi_fail(c, EB_ERR_INVALID_ARG, "yp / out must be 16-byte aligned");
+  if (!ebi_aligned16(yp) || !ebi_aligned16(out) || !ebi_aligned16(residual))
+    return ebi_fail(c, EB_ERR_INVALID_ARG, "yp / out / residual must be 16-byte aligned");
   if (bp.n_tok == 0) return EB_OK;
   const combine_fn* table = combine_table(std::make_integer_sequence<int, kMaxSlots>());
   cudaStream_t st = (cudaStream_t)stream;
@@ -86,7 +105,7 @@ extern "C" eb_status eb_combine(eb_ctx* c, void* stream, const eb_batch* batch, 
   const int vec = c->cfg.H / 8;
   const int team = vec <= 32 ? 32 : vec <= 64 ? 64 : vec <= 128 ? 128 : 256, tpb = kThreads / team;
   ebi_launch(table[KS], dim3((bp.n_tok + tpb - 1) / tpb), dim3(kThreads), 0, st, bp.n_tok, c->cfg.H, c->cfg.K, team,
-             (const uint4*)yp, pos, topk_w, (uint4*)out);
+             (const uint4*)yp, pos, topk_w, (const uint4*)residual, (uint4*)out);
   EB_LAUNCH_CHECK(c, "combine");
   return EB_OK;
 }

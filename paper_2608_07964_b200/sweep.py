@@ -51,17 +51,10 @@ def ep_size_sweep(args, dev, weights):
             for name, pol in (("max", B.POLICY_MAXUTIL), ("cum", B.POLICY_CUMUTIL), ("diff", B.POLICY_DIFFPEAK)):
                 res[name] = driver.idle_fractions(driver.run_load_trace(step, wl.tok_off, wl.L, wl.m, pol, logits_of), D)
             lock = driver.idle_fractions(driver.run_load_trace(step, wl.tok_off, wl.L, wl.N, B.POLICY_ALL, logits_of), D)
-            # per (micro-batch, layer) peak device from the routed loads
-            peaks = {}
-            for l in range(wl.L):
-                for j in range(wl.N):
-                    step.logits[wl.tok_off[j]:wl.tok_off[j + 1]].copy_(logits_of(j, l))
-                step.eb_route(B.Batch(wl.tok_off, [l] * wl.N))
-                loads = step.mb_load[:wl.N].cpu().tolist()
-                for j in range(wl.N):
-                    peaks[(j, l)] = max(range(D), key=lambda d: (loads[j][d], -d))
-            same2 = sum(peaks[(j, l)] == peaks[(j, l + 1)] for j in range(wl.N) for l in range(wl.L - 1))
-            same3 = sum(peaks[(j, l)] == peaks[(j, l + 1)] == peaks[(j, l + 2)] for j in range(wl.N) for l in range(wl.L - 2))
+            # how often a micro-batch's workload keeps its peak device over 2 and 3 consecutive layers
+            loads = driver.routed_loads(step, wl.tok_off, wl.L, logits_of)
+            same2 = sum(driver.same_peak_windows(loads[j], 2)[0] for j in range(wl.N))
+            same3 = sum(driver.same_peak_windows(loads[j], 3)[0] for j in range(wl.N))
             lines.append(f"| {s} | {D} | {wl.T} | {res['max']['idle_cross_layer']:.3f} | {res['cum']['idle_cross_layer']:.3f} | "
                          f"{res['diff']['idle_cross_layer']:.3f} | {res['max']['idle_each_alone']:.3f} | {lock['idle_cross_layer']:.3f} | "
                          f"{same2}/{wl.N * (wl.L - 1)} | {same3}/{wl.N * (wl.L - 2)} |")
@@ -121,6 +114,23 @@ def schedule_latency_report(args, dev):
     return lines
 
 
+def front_end_steps(args, dev, weights):
+    """A few whole steps at N = 4, 8, 16 micro-batches of 16 tokens (the fused permutation path), for a launch
+    list: the scheduling and permutation kernels' durations are read off a profiler's per-launch times."""
+    for N in (4, 8, 16):
+        wl = synth.workload_c5(N, 16, 1.0)
+        step = B.from_workload(wl, device=dev)
+        step.bind_weights(*weights)
+        step.logits[:wl.T_tot].copy_(synth.packed_logits(wl, device=dev))
+        step.x[:wl.T_tot].copy_(synth.packed_hidden(wl, device=dev))
+        batch = B.Batch(wl.tok_off, wl.layers)
+        ms = timed_ms(lambda: step.eb_step(batch, wl.m), reps=5, warm=3)
+        assert step.device_status() == 0
+        print(f"N={N} m={wl.m} step {ms:.3f} ms", flush=True)
+        step.close()
+    return []
+
+
 def m_sweep(args, dev, weights):
     """Minimum combination size sweep (the paper's micro-batching ablation): for every micro-batch count N and
     every m from 1 to N, whole-run under-utilisation of Algorithm 1 under the three policies, the number of steps,
@@ -160,6 +170,7 @@ def main(argv=None):
     ap.add_argument("--latency", action="store_true", help="emulated expert-parallel latency of whole runs")
     ap.add_argument("--sched", action="store_true", help="time of one scheduling call per policy")
     ap.add_argument("--msweep", action="store_true", help="minimum combination size sweep")
+    ap.add_argument("--front", action="store_true", help="a few steps at N = 4, 8, 16 for a launch list of the small kernels")
     args = ap.parse_args(argv)
     dev = "cuda:0"
     if args.sched:
@@ -176,6 +187,9 @@ def main(argv=None):
         return 0
     base = synth.workload_c5(2, 16, 0.0)
     weights = tuple(synth.all_weights(base, k, dev) for k in ("gate", "up", "down"))
+    if args.front:
+        front_end_steps(args, dev, weights)
+        return 0
     if args.msweep:
         text = "\n".join(m_sweep(args, dev, weights)) + "\n"
         if args.out:

@@ -27,7 +27,7 @@ def test_header_symbols_are_exported_and_bound():
 def test_struct_layouts_match_the_header():
     assert ctypes.sizeof(binding.EbSchedResult) == 96
     assert binding.EbSchedResult.util_num.offset == 80
-    assert ctypes.sizeof(binding.EbStepBuffers) == 15 * 8
+    assert ctypes.sizeof(binding.EbStepBuffers) == 16 * 8
     assert ctypes.sizeof(binding.EbConfig) == 48
     text = open(os.path.join(ROOT, "include", "eb.h")).read()
     for name in ("EB_MAX_MB", "EB_MAX_D", "EB_META_LEN", "EB_HOST_SLOTS"):
