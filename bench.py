@@ -41,7 +41,9 @@ UNIT = "tokens/s"
 # dram__bytes_write.sum) over the algorithmic bytes of the captured launch.  The captures ran on cut-down cases
 # of the same shapes (a full-size capture would hold tens of GB); traffic grows in proportion to the weight
 # bytes streamed, so a full launch is that ratio times its own algorithmic bytes.
-NCU_TRAFFIC_RATIO = {}
+NCU_TRAFFIC_RATIO = {"c4": 4.112702 / 3.909091, "c4small": 4.112702 / 3.909091,          # captured on c4small
+                     "c2": 1.496576 / 1.487012, "c2small": 1.496576 / 1.487012,          # captured on c2small
+                     "c3init": 1.175985 / 1.101005, "c3initsmall": 1.175985 / 1.101005}  # captured on c3initsmall
 
 
 def measured_peaks():
