@@ -86,7 +86,7 @@ static size_t carve(eb_ctx* c, char* base) {
   c->group_size = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
   c->pgroup = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
   c->pslots = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
-  c->pcost = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
+  c->prank = (int4*)take(sizeof(int4) * (size_t)gcap);
   c->order = (int32_t*)take(sizeof(int32_t) * (size_t)gcap);
   c->tile_pref = (int32_t*)take(sizeof(int32_t) * (size_t)(gcap + 1));
   c->work_count = (int32_t*)take(sizeof(int32_t) * 16);

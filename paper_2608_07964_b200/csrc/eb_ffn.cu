@@ -495,31 +495,52 @@ __device__ __forceinline__ bool merged_class(const ModelParams& mp, const int* d
   return mx <= kMergeMaxRows;
 }
 
-// Block-wide exclusive scan of one value per thread (1024 threads); returns the exclusive prefix and
-// leaves the block total in *total.  Ends with a barrier, so s_warp may be reused right away.
-__device__ __forceinline__ long long block_scan_excl(long long v, long long* s_warp, long long* total) {
+// Cost classes of the tiles: class c holds the positions whose tiles have 32 (c + 1) columns.
+constexpr int kClasses = kTileRows / 32;
+
+// Block-wide exclusive scan (1024 threads) of one value per thread that belongs to one of kClasses classes:
+// returns the sum of the values of the same class in the threads before this one, and adds every class's
+// block total to total[].  A value packs two counters (low / high 32 bits).  Ends with a barrier.
+__device__ __forceinline__ long long block_scan_by_class(int cls, long long v, long long (*s_warp)[kClasses],
+                                                         long long* total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  long long incl = v;
+  long long incl[kClasses];
+#pragma unroll
+  for (int c = 0; c < kClasses; ++c) incl[c] = c == cls ? v : 0;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    long long n = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += n;
+#pragma unroll
+    for (int c = 0; c < kClasses; ++c) {
+      const long long n = __shfl_up_sync(0xffffffffu, incl[c], o);
+      if (lane >= o) incl[c] += n;
+    }
   }
-  if (lane == 31) s_warp[warp] = incl;
+  if (lane == 31) {
+#pragma unroll
+    for (int c = 0; c < kClasses; ++c) s_warp[warp][c] = incl[c];
+  }
   __syncthreads();
   if (warp == 0) {
-    long long wv = s_warp[lane], wi = wv;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      long long n = __shfl_up_sync(0xffffffffu, wi, o);
-      if (lane >= o) wi += n;
+    for (int c = 0; c < kClasses; ++c) {
+      const long long wv = s_warp[lane][c];
+      long long wi = wv;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const long long n = __shfl_up_sync(0xffffffffu, wi, o);
+        if (lane >= o) wi += n;
+      }
+      s_warp[lane][c] = wi - wv;
+      if (lane == 31) s_warp[32][c] = wi;
     }
-    s_warp[lane] = wi - wv;
-    if (lane == 31) s_warp[32] = wi;
   }
   __syncthreads();
-  const long long excl = s_warp[warp] + incl - v;
-  *total = s_warp[32];
+  long long excl = 0;
+#pragma unroll
+  for (int c = 0; c < kClasses; ++c) {
+    if (c == cls) excl = s_warp[warp][c] + incl[c] - v;
+    total[c] += s_warp[32][c];
+  }
   __syncthreads();
   return excl;
 }
@@ -527,13 +548,13 @@ __device__ __forceinline__ long long block_scan_excl(long long v, long long* s_w
 // plan: per position i of the processing order (requested group range), the group, its tile count and
 // cost class; then the positions that own tiles are listed by cost class (widest tiles first, processing
 // order inside a class) with the exclusive scan of their tile counts.  Widest-first order lets the
-// expert kernel deal its tiles out in rounds of near-equal cost.
+// expert kernel deal its tiles out in rounds of near-equal cost.  One scan carries all classes at once.
 __global__ void __launch_bounds__(1024)
 plan_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t* __restrict__ step_meta, int device,
-            int nt1, int nt2, int32_t* __restrict__ pgroup, int32_t* __restrict__ pslots, int32_t* __restrict__ pcost,
+            int nt1, int nt2, int32_t* __restrict__ pgroup, int32_t* __restrict__ pslots, int4* __restrict__ prank,
             int32_t* __restrict__ order, int32_t* __restrict__ tile_pref, int32_t* __restrict__ work_count) {
   EB_GRID_DEP_SYNC();
-  __shared__ long long s_warp[33];
+  __shared__ long long s_warp[33][kClasses];
   __shared__ int s_dev_off[EB_MAX_D + 1];
   const int tid = threadIdx.x;
   if (tid <= mp.D) s_dev_off[tid] = mp.dev_off[tid];
@@ -543,7 +564,12 @@ plan_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t
   const int ng = g1 - g0;
   const int nl = step_meta[2];
   __syncthreads();
-  unsigned classes = 0;   // bit c: some position has tiles of 32 (c + 1) columns
+  // pass 1: tiles and class of every position; its rank and tile prefix inside its class
+  long long total[kClasses];   // low 32 bits: positions of the class, high 32 bits: their tiles
+#pragma unroll
+  for (int c = 0; c < kClasses; ++c) total[c] = 0;
+  int my_cls = -1;             // of the position this thread handled in the last chunk (the only one, as a rule)
+  long long my_at = 0;
   for (int b = 0; b < ng; b += 1024) {
     const int i = b + tid;
     int tiles = 0, cols = 0;
@@ -563,33 +589,53 @@ plan_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t
         tiles = group_tiles(rows);
         cols = group_cols(rows);
       }
-      pcost[i] = tiles | (cols << 20);
     }
-    for (int c = 0; c < kTileRows / 32; ++c)
-      if (__syncthreads_or(tiles > 0 && cols == 32 * (c + 1))) classes |= 1u << c;
+    const int cls = tiles > 0 ? cols / 32 - 1 : -1;
+    long long before[kClasses];
+#pragma unroll
+    for (int c = 0; c < kClasses; ++c) before[c] = total[c];
+    const long long excl = block_scan_by_class(cls, tiles > 0 ? (1LL | ((long long)tiles << 32)) : 0, s_warp, total);
+    my_cls = cls;
+    my_at = 0;
+#pragma unroll
+    for (int c = 0; c < kClasses; ++c)
+      if (c == cls) my_at = before[c] + excl;
+    // more than one chunk of positions: parked until the class bases are known (read back by the same thread)
+    if (ng > 1024 && i < ng) prank[i] = make_int4(cls, (int)(my_at & 0xffffffffLL), (int)(my_at >> 32), 0);
   }
-  long long carry = 0;   // low 32 bits: positions listed so far, high 32 bits: their tiles
-  for (int c = kTileRows / 32 - 1; c >= 0; --c) {
-    if (!((classes >> c) & 1u)) continue;
-    for (int b = 0; b < ng; b += 1024) {
-      const int i = b + tid;
-      long long v = 0;
+  // class bases: widest class first
+  long long base[kClasses];
+  long long run = 0;
+#pragma unroll
+  for (int c = kClasses - 1; c >= 0; --c) {
+    base[c] = run;
+    run += total[c];
+  }
+  const int n_listed = (int)(run & 0xffffffffLL), nt = (int)(run >> 32);
+  // pass 2: place every position that owns tiles
+  for (int b = 0; b < ng; b += 1024) {
+    const int i = b + tid;
+    int cls = my_cls, rank = (int)(my_at & 0xffffffffLL), tpref = (int)(my_at >> 32);
+    if (ng > 1024) {
+      cls = -1;
       if (i < ng) {
-        const int pc = pcost[i];
-        if ((pc & 0xfffff) > 0 && (pc >> 20) == 32 * (c + 1)) v = 1LL | ((long long)(pc & 0xfffff) << 32);
+        const int4 v = prank[i];
+        cls = v.x;
+        rank = v.y;
+        tpref = v.z;
       }
-      long long total;
-      const long long excl = block_scan_excl(v, s_warp, &total);
-      if (v) {
-        const long long at = carry + excl;
-        order[(int)(at & 0xffffffffLL)] = i;
-        tile_pref[(int)(at & 0xffffffffLL)] = (int)(at >> 32);
-      }
-      carry += total;
+    }
+    if (cls >= 0) {
+      long long b2 = 0;
+#pragma unroll
+      for (int c = 0; c < kClasses; ++c)
+        if (c == cls) b2 = base[c];
+      const int at = (int)(b2 & 0xffffffffLL) + rank;
+      order[at] = i;
+      tile_pref[at] = (int)(b2 >> 32) + tpref;
     }
   }
   if (tid == 0) {
-    const int n_listed = (int)(carry & 0xffffffffLL), nt = (int)(carry >> 32);
     tile_pref[n_listed] = nt;
     work_count[0] = nt * nt1;
     work_count[1] = nt * nt2;
@@ -610,8 +656,12 @@ fill_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t
             const int32_t* __restrict__ tile_pref, const int32_t* __restrict__ work_count, int nt1, int nt2, int max1,
             int max2, int4* __restrict__ work1, int4* __restrict__ work2, int2* __restrict__ slots) {
   EB_GRID_DEP_SYNC();
+  extern __shared__ int s_pref[];   // tile_pref staged once per block: the binary search below then stays on chip
   const int n_listed = work_count[5];
   const int cnt1 = work_count[0], total = cnt1 + work_count[1];
+  if ((int)(blockIdx.x * blockDim.x) >= total) return;
+  for (int i = threadIdx.x; i <= n_listed; i += blockDim.x) s_pref[i] = tile_pref[i];
+  __syncthreads();
   for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
     const int list = idx >= cnt1 ? 1 : 0, local = idx - (list ? cnt1 : 0);
     const int nt = list ? nt2 : nt1;
@@ -620,16 +670,16 @@ fill_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t
     int lo = 0, hi = n_listed - 1;
     while (lo < hi) {
       int mid = (lo + hi + 1) >> 1;
-      if (tile_pref[mid] <= t_index) lo = mid; else hi = mid - 1;
+      if (s_pref[mid] <= t_index) lo = mid; else hi = mid - 1;
     }
-    const int t_g = tile_pref[lo + 1] - tile_pref[lo];
-    const int rem = local - tile_pref[lo] * nt;
+    const int t_g = s_pref[lo + 1] - s_pref[lo];
+    const int rem = local - s_pref[lo] * nt;
     const int n = rem / t_g, m = rem % t_g;
     const int pos = order[lo], g = pgroup[pos], n_slots = pslots[pos];
     int4 it;
     if (n_slots >= 0) {
       // tile m of a merged class holds the next 16 slots of the class, replicas in device order
-      const int base = kMergeSlots * (tile_pref[lo] + m);
+      const int base = kMergeSlots * (s_pref[lo] + m);
       const int first = kMergeSlots * m, n_here = min(kMergeSlots, n_slots - first);
       if (list == 0 && n == 0) {
         int c = 0;   // slots before the current replica
@@ -774,11 +824,12 @@ eb_status ebi_ffn_run(eb_ctx* c, cudaStream_t st, const void* xp, const int32_t*
   {
     KernelTimer timer(c, EBK_FFN_PLAN, st);
     ebi_launch(plan_kernel, dim3(1), dim3(1024), 0, st, c->mp, group_off, step_meta, (int)device, nt1, nt2, c->pgroup, c->pslots,
-               c->pcost, c->order, c->tile_pref, c->work_count);
+               c->prank, c->order, c->tile_pref, c->work_count);
   }
   {
     KernelTimer timer(c, EBK_FFN_FILL, st);
-    ebi_launch(fill_kernel, dim3(c->num_sms), dim3(256), 0, st, c->mp, group_off, group_w, (const int32_t*)c->pgroup,
+    ebi_launch(fill_kernel, dim3(c->num_sms), dim3(256), sizeof(int) * (size_t)(ebi_groups_cap(c) + 1), st, c->mp, group_off, group_w,
+               (const int32_t*)c->pgroup,
                (const int32_t*)c->pslots, (const int32_t*)c->order, (const int32_t*)c->tile_pref,
                (const int32_t*)c->work_count, nt1, nt2, c->max_work1, c->max_work2, c->work1, c->work2, c->slots);
   }

@@ -75,7 +75,7 @@ struct eb_ctx {
   int32_t* group_size = nullptr;   // [G_cap]
   int32_t* pgroup = nullptr;       // [G_cap] group at each position of the processing order
   int32_t* pslots = nullptr;       // [G_cap] 16-row slots of the merged shared-expert class of the position, -1 otherwise
-  int32_t* pcost = nullptr;        // [G_cap] tiles | columns << 20 of the position
+  int4* prank = nullptr;           // [G_cap] (cost class, rank and tiles before it inside the class) when a plan has more than 1024 positions
   int32_t* order = nullptr;        // [G_cap] positions that own tiles, widest tiles first
   int32_t* tile_pref = nullptr;    // [G_cap + 1] tiles before each entry of `order`
   int32_t* work_count = nullptr;   // [16]: tile counts of the two lists, group range, layers, device filter

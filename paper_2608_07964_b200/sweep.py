@@ -1,6 +1,6 @@
 """Skew / micro-batch sweep on the 64-expert, top-6, hidden-2048 shape (8 layers, 8 virtual devices).
 
-    python -m paper_2608_07964_b200.sweep [--out results.md] [--policy 0] [--ep | --msweep | --latency | --sched]
+    python -m paper_2608_07964_b200.sweep [--out results.md] [--policy 0] [--ep | --msweep | --latency | --sched | --whole | --front]
 
 For every point (Zipf s, micro-batch count N, tokens per micro-batch T) it reports
   * whole-run under-utilisation 1 - u of Algorithm 1 driven on the GPU (route + schedule every
@@ -114,6 +114,47 @@ def schedule_latency_report(args, dev):
     return lines
 
 
+def whole_run_report(args, dev):
+    """Whole Algorithm-1 runs executed in full on the benchmark shapes (every step one eb_step with the residual
+    added in place): device time and token-layers per second for cross-layer scheduling (MaxUtil, m = ceil(0.75 N)),
+    for lock-step execution (all micro-batches jointly, layer by layer) and with each step replayed from a CUDA
+    graph; plus the emulated expert-parallel latency (per step the slowest virtual device's expert pass) and the
+    time-based idle fraction of cross-layer scheduling, lock-step execution and every workload alone."""
+    lines = ["| shape | policy | steps | whole-run ms | token-layers/s | same, steps replayed from CUDA graphs | emulated EP latency ms | time idle |",
+             "|---|---|---|---|---|---|---|---|"]
+    for name in ("c3", "c4"):
+        wl = synth.workload(name)
+        bias = synth.zipf_bias(wl)
+        step = B.from_workload(wl, device=dev)
+        weights = tuple(synth.all_weights(wl, k, dev) for k in ("gate", "up", "down"))
+        step.bind_weights(*weights)
+        logits_of = lambda j, l: synth.logits_for(wl, j, l, dev, bias)
+        # random-weight blocks without the normalisation layers of a real model grow the hidden state layer by
+        # layer; a twentieth of the unit scale keeps 26 to 32 of them finite (timing does not depend on the values)
+        x0 = (torch.cat([synth.hidden_for(wl, j, 0, dev) for j in range(wl.N)], 0).float() * 0.05).to(torch.bfloat16)
+        for label, m, pol in (("cross-layer MaxUtil", wl.m, B.POLICY_MAXUTIL), ("lock-step", wl.N, B.POLICY_ALL)):
+            driver.run_full(step, wl.tok_off, wl.L, m, pol, logits_of, x0)                       # warm
+            r = driver.run_full(step, wl.tok_off, wl.L, m, pol, logits_of, x0)
+            graphs = driver.StepGraphs(step, wl.tok_off, capacity=4096)
+            driver.run_full(step, wl.tok_off, wl.L, m, pol, logits_of, x0, graphs=graphs)       # captures
+            rg = driver.run_full(step, wl.tok_off, wl.L, m, pol, logits_of, x0, graphs=graphs)  # replays
+            same = torch.equal(r["x"].view(torch.int16), rg["x"].view(torch.int16))
+            finite = bool(torch.isfinite(r["x"].float()).all())
+            assert same and finite, (label, same, finite)
+            lat = driver.run_emulated_latency(step, wl.tok_off, wl.L, wl.D, m, pol, logits_of, x0)
+            lines.append(f"| {name} | {label} (m = {m}) | {len(r['steps'])} | {r['ms']:.1f} | {r['token_layers'] / r['ms'] * 1e3:.3e} | "
+                         f"{rg['ms']:.1f} ms, {rg['token_layers'] / rg['ms'] * 1e3:.3e} | {lat['latency_ms']:.2f} | {lat['idle_time']:.3f} |")
+            print(lines[-1], flush=True)
+        lat = driver.run_emulated_latency(step, wl.tok_off, wl.L, wl.D, 1, B.POLICY_ALL, logits_of, x0, alone=True)
+        lines.append(f"| {name} | every workload alone | {lat['steps']} | - | - | - | {lat['latency_ms']:.2f} | {lat['idle_time']:.3f} |")
+        print(lines[-1], flush=True)
+        assert step.device_status() == 0
+        step.close()
+        del weights
+        torch.cuda.empty_cache()
+    return lines
+
+
 def front_end_steps(args, dev, weights):
     """A few whole steps at N = 4, 8, 16 micro-batches of 16 tokens (the fused permutation path), for a launch
     list: the scheduling and permutation kernels' durations are read off a profiler's per-launch times."""
@@ -170,11 +211,18 @@ def main(argv=None):
     ap.add_argument("--latency", action="store_true", help="emulated expert-parallel latency of whole runs")
     ap.add_argument("--sched", action="store_true", help="time of one scheduling call per policy")
     ap.add_argument("--msweep", action="store_true", help="minimum combination size sweep")
+    ap.add_argument("--whole", action="store_true", help="whole Algorithm-1 runs executed in full on the benchmark shapes")
     ap.add_argument("--front", action="store_true", help="a few steps at N = 4, 8, 16 for a launch list of the small kernels")
     args = ap.parse_args(argv)
     dev = "cuda:0"
     if args.sched:
         text = "\n".join(schedule_latency_report(args, dev)) + "\n"
+        if args.out:
+            with open(args.out, "w") as f:
+                f.write(text)
+        return 0
+    if args.whole:
+        text = "\n".join(whole_run_report(args, dev)) + "\n"
         if args.out:
             with open(args.out, "w") as f:
                 f.write(text)
