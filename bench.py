@@ -400,6 +400,18 @@ def measure(args, wl, device, local, dist, full):
     res["idle"] = idle_report(step, batch, wl, sched, B) if dist is None and not args.no_idle else None
 
     res["cpu"] = None
+    if not full and dist is None and not args.no_cpu_baseline and wl.name in ("c1", "c2"):
+        # small shapes: the oracle's whole step with all host threads and with one (a few seconds each)
+        from threadpoolctl import threadpool_limits
+        get = lazy_cpu_weights(wl, device)
+        lg, xx = logits.cpu().numpy(), x.float().cpu().numpy()
+        oracle_step_sample(wl, lg, xx, get, 1.0)          # stages the sampled weights on the host
+        r = oracle_step_sample(wl, lg, xx, get, 4.0)
+        with threadpool_limits(limits=1):
+            r1 = oracle_step_sample(wl, lg, xx, get, 4.0)
+        res["cpu"] = dict(value=r["tokens"] / r["seconds"], unit=UNIT, cores=cpu_threads(), kind="oracle",
+                          rows=f"{r['rows']} of {r['rows_total']}", single_thread_value=r1["tokens"] / r1["seconds"],
+                          single_thread_rows=f"{r1['rows']} of {r1['rows_total']}")
     if full and dist is None and not args.no_cpu_baseline:
         get = lazy_cpu_weights(wl, device)
         lg, xx = logits.cpu().numpy(), x.float().cpu().numpy()
@@ -429,7 +441,7 @@ def compact(res, peaks):
                 expert_pass_tflops=ex["ffn"]["tflops"], expert_pass_frac_burst=ex["ffn"]["frac_tensor_peak"],
                 expert_pass_frac_sustained=ex["ffn"]["frac_tensor_sustained"], expert_pass_frac_hbm=ex["ffn"]["frac_hbm"],
                 front_end_ms=ex["front_end_ms"], gather_gbs=ex["permute_gather"]["gbs"], combine_gbs=ex["combine"]["gbs"],
-                idle=res["idle"])
+                idle=res["idle"], cpu_baseline=res["cpu"])
 
 
 def run_ours(args, wl):
