@@ -11,7 +11,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 @pytest.mark.gpu
 def test_bench_line_has_the_contract_keys():
-    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--workload", "c1", "--steps", "3", "--warmup", "3"],
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--workload", "c1", "--steps", "3", "--warmup", "3", "--sustain-s", "0.3"],
                        capture_output=True, text=True, timeout=600)
     assert r.returncode == 0, r.stderr[-800:]
     lines = [l for l in r.stdout.strip().splitlines() if l.startswith("{")]
@@ -31,3 +31,8 @@ def test_bench_line_has_the_contract_keys():
     cpu = d["cpu_baseline"]
     assert cpu["kind"] == "oracle" and cpu["value"] > 0 and cpu["cores"] >= 1 and cpu["sample"]
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
+    # both expert launches with their own algorithmic work and roofline entry; the sustained-loop leg
+    for k in ("ffn_gateup", "ffn_down"):
+        e = d["detail"]["launches"][k]
+        assert e["ms"] > 0 and e["algorithmic_bytes"] > 0 and e["algorithmic_flops"] > 0 and e["bound"] in ("hbm", "tensor")
+    assert d["detail"]["sustained"]["ms_per_step"] > 0 and d["detail"]["sustained"]["steps"] >= 10
