@@ -448,13 +448,16 @@ def test_argument_errors_return_codes():
 
 
 # ----------------------------------------------------------------------------------- CTA-pair tiles
-def test_group_sizes_around_the_pair_tile_boundaries():
-    """Exact group sizes on both sides of every rule that sends a group to 128-row tiles on single CTAs
-    or to 256-row tiles on CTA pairs; every row of every group is compared."""
-    B = _binding()
-    sizes = [129, 256, 257, 384, 385, 512, 513, 640, 100, 1, 128, 0, 300, 768]
+@pytest.mark.parametrize("H,I", [(192, 328), (520, 264)])
+def test_group_sizes_around_the_tile_boundaries(H, I):
+    """Exact group sizes on both sides of every place where the expert kernel's tiling changes: the 32-row
+    steps of a tile's column count, the 128 rows one CTA of a pair loads, and the 256-row limit at which a group
+    is cut into two, three, four nearly equal tiles; output widths that end inside the first CTA's half of an
+    output tile, inside the second, and just past a whole tile.  Every row of every group is compared."""
+    sizes = [1, 16, 31, 32, 33, 63, 64, 65, 96, 97, 128, 129, 160, 255, 256, 257, 288, 511, 512, 513, 767, 768, 769,
+             1000, 0]
     E = len(sizes)
-    wl = synth.Workload(name="pairs", L=1, E=E, K=1, S=0, H=192, I=328, D=2, mapping="mod", N=1, T=sum(sizes),
+    wl = synth.Workload(name="tiles", L=1, E=E, K=1, S=0, H=H, I=I, D=2, mapping="mod", N=1, T=sum(sizes),
                         zipf_s=0.0)
     store = Hn.WeightStore(wl)
     case = Hn.make_case(wl)
