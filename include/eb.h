@@ -293,6 +293,13 @@ eb_status eb_check_permutation(eb_ctx* ctx, void* stream, const eb_batch* batch,
                                const int32_t* row_src, const int32_t* pos, const int32_t* step_meta,
                                int32_t* out_errors);
 
+/* The workspace regions (permutation tables, tile lists, intermediate activations) are separated by guard
+ * areas of 256 bytes that eb_set_workspace fills with a pattern and no kernel ever writes.  This call counts
+ * the guard bytes that no longer hold the pattern (*out_bad, host; 0 = intact) and synchronises the stream:
+ * a kernel that wrote past the end of its region shows up here instead of silently corrupting its neighbour.
+ * The paper has no counterpart: a debugging aid for boxes without a memory checker. */
+eb_status eb_check_workspace_guards(eb_ctx* ctx, void* stream, int32_t* out_bad);
+
 /* Exercises the bounded wait used by the expert kernels without any fault: one CTA waits on a
  * barrier that nothing arrives on, for at most `limit_cycles` SM cycles (1 .. 2e9), then gives up,
  * records EB_ERR_TIMEOUT in the context status word and returns normally.  *out_gave_up (host) is

@@ -48,7 +48,7 @@ SYMBOLS = ["eb_create", "eb_destroy", "eb_bind_weights", "eb_workspace_bytes", "
            "eb_rows_capacity", "eb_groups_capacity", "eb_route", "eb_schedule", "eb_permute",
            "eb_expert_ffn_grouped", "eb_expert_ffn_device", "eb_combine", "eb_combine_residual", "eb_step", "eb_step_host",
            "eb_step_host_submit", "eb_step_host_wait",
-           "eb_permute_noalloc", "eb_selftest_bounded_wait", "eb_check_permutation",
+           "eb_permute_noalloc", "eb_selftest_bounded_wait", "eb_check_permutation", "eb_check_workspace_guards",
            "eb_device_status", "eb_num_kernels", "eb_kernel_name", "eb_set_timing", "eb_kernel_ms",
            "eb_launch_count", "eb_status_string", "eb_last_error"]
 
@@ -91,6 +91,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.eb_permute_noalloc.argtypes = [C.POINTER(EbConfig), vp, C.POINTER(EbBatch), vp, vp, vp, vp, vp, vp, vp, vp, vp,
                                        C.c_char_p, C.c_size_t]
     lib.eb_check_permutation.argtypes = [vp, vp, C.POINTER(EbBatch), vp, vp, vp, vp, vp, vp, vp, C.POINTER(i32)]
+    lib.eb_check_workspace_guards.argtypes = [vp, vp, C.POINTER(i32)]
     lib.eb_selftest_bounded_wait.argtypes = [vp, vp, C.c_int64, C.POINTER(i32)]
     lib.eb_device_status.argtypes = [vp, C.POINTER(i32)]
     lib.eb_num_kernels.argtypes = []
@@ -337,6 +338,12 @@ class MoEStep:
                                                   self.topk_idx.data_ptr(), self.group_off.data_ptr(),
                                                   self.group_w.data_ptr(), self.row_src.data_ptr(), self.pos.data_ptr(),
                                                   self.step_meta.data_ptr(), C.byref(v)))
+        return v.value
+
+    def check_workspace_guards(self) -> int:
+        """Guard bytes between the workspace regions that no longer hold their pattern (0 = intact)."""
+        v = C.c_int32(-1)
+        self._check(self.lib.eb_check_workspace_guards(self.ctx, _stream(), C.byref(v)))
         return v.value
 
     def selftest_bounded_wait(self, limit_cycles: int = 2_000_000) -> int:

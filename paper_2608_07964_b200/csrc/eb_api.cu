@@ -67,13 +67,21 @@ eb_status ebi_make_batch(eb_ctx* c, const eb_batch* b, BatchParams* out) {
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+constexpr size_t kGuardBytes = 256;
+constexpr int kGuardByte = 0xA5;
+
 // Lays the workspace regions out; with base == nullptr only the total size is computed.
 static size_t carve(eb_ctx* c, char* base) {
   const eb_config& g = c->cfg;
   size_t off = 0;
+  c->n_guards = 0;
   auto take = [&](size_t bytes) {
     char* p = base ? base + off : nullptr;
     off = align_up(off + bytes, 256);
+    // a guard of kGuardBytes after every region: filled with a pattern by eb_set_workspace, never written by any
+    // kernel, checked by eb_check_workspace_guards
+    if (c->n_guards < EB_MAX_GUARDS) c->guard_off[c->n_guards++] = off;
+    off += kGuardBytes;
     return p;
   };
   c->max_chunks = (g.max_tokens + 31) / 32 + EB_MAX_MB;
@@ -208,6 +216,8 @@ extern "C" eb_status eb_set_workspace(eb_ctx* c, void* dev_ptr, size_t bytes) {
   c->ws = dev_ptr;
   c->ws_bytes = bytes;
   carve(c, (char*)dev_ptr);
+  for (int i = 0; i < c->n_guards; ++i)
+    EB_CUDA(c, cudaMemset((char*)dev_ptr + c->guard_off[i], kGuardByte, kGuardBytes));
   return EB_OK;
 }
 
@@ -329,6 +339,37 @@ extern "C" eb_status eb_device_status(eb_ctx* c, int32_t* out_status) {
   EB_CUDA(c, cudaDeviceSynchronize());
   EB_CUDA(c, cudaMemcpy(out_status, c->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost));
   EB_CUDA(c, cudaMemset(c->d_status, 0, sizeof(int32_t)));
+  return EB_OK;
+}
+
+namespace {
+struct GuardList {
+  int n;
+  unsigned long long off[EB_MAX_GUARDS];
+};
+__global__ void check_guards_kernel(const unsigned char* ws, GuardList g, int* bad) {
+  int n = 0;
+  for (int i = 0; i < g.n; ++i)
+    for (int b = threadIdx.x; b < (int)kGuardBytes; b += blockDim.x)
+      if (ws[g.off[i] + b] != (unsigned char)kGuardByte) ++n;
+  if (n) atomicAdd(bad, n);
+}
+}  // namespace
+
+extern "C" eb_status eb_check_workspace_guards(eb_ctx* c, void* stream, int32_t* out_bad) {
+  if (!c || !out_bad) return EB_ERR_INVALID_ARG;
+  if (eb_status ds = ebi_check_device(c)) return ds;
+  if (!c->ws) return ebi_fail(c, EB_ERR_WORKSPACE, "no workspace set");
+  cudaStream_t st = (cudaStream_t)stream;
+  GuardList g;
+  g.n = c->n_guards;
+  for (int i = 0; i < c->n_guards; ++i) g.off[i] = c->guard_off[i];
+  int* d_bad = c->work_count + 14;   // scratch word of the workspace
+  EB_CUDA(c, cudaMemsetAsync(d_bad, 0, sizeof(int), st));
+  check_guards_kernel<<<1, 256, 0, st>>>((const unsigned char*)c->ws, g, d_bad);
+  EB_LAUNCH_CHECK(c, "check_workspace_guards");
+  EB_CUDA(c, cudaMemcpyAsync(out_bad, d_bad, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  EB_CUDA(c, cudaStreamSynchronize(st));
   return EB_OK;
 }
 

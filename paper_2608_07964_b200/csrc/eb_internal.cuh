@@ -14,6 +14,8 @@
 
 typedef __nv_bfloat16 bf16;
 
+enum { EB_MAX_GUARDS = 24 };
+
 // Kernel ids for the optional per-kernel event timing.
 enum EbKernel {
   EBK_ROUTE = 0,
@@ -70,6 +72,8 @@ struct eb_ctx {
   // workspace carve-up
   void* ws = nullptr;
   size_t ws_bytes = 0;
+  int n_guards = 0;                // guard areas between the regions below (debugging aid)
+  size_t guard_off[EB_MAX_GUARDS] = {};
   int32_t* chunk_hist = nullptr;   // [max_chunks][E]
   int32_t* chunk_base = nullptr;   // [max_chunks][E]
   int32_t* group_size = nullptr;   // [G_cap]

@@ -63,6 +63,7 @@ def _full_step(case, store, m, policy=O.POLICY_MAXUTIL, pool_mask=None, check_ff
     torch.cuda.synchronize()
     assert step.device_status() == 0
     assert step.check_permutation(batch) == 0
+    assert step.check_workspace_guards() == 0, "a kernel wrote past the end of its workspace region"
 
     ref = Hn.oracle_front(case, pool, m, policy)
     Hn.check_front(step, case, ref, n_mb)
@@ -536,6 +537,20 @@ def test_step_replayed_from_a_cuda_graph_matches_eager():
         assert step.sched_result()["run_mask"] == mask_replayed
         assert torch.equal(step.out[:T], replayed)
     assert step.device_status() == 0
+
+
+def test_workspace_guards_detect_a_write_past_a_region():
+    B = _binding()
+    wl = synth.workload("c1")
+    step = B.from_workload(wl)
+    assert step.check_workspace_guards() == 0
+    # the first guard follows the first region (per-chunk histograms): overwrite three of its bytes from the host side
+    first_region = 4 * ((wl.T_tot + 31) // 32 + B.EB_MAX_MB) * wl.E
+    off = (first_region + 255) // 256 * 256
+    step.workspace[off + 5:off + 8] = 0
+    assert step.check_workspace_guards() == 3
+    step.workspace[off + 5:off + 8] = 0xA5
+    assert step.check_workspace_guards() == 0
 
 
 def test_device_side_checker_flags_corrupted_tables():
