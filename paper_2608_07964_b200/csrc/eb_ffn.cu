@@ -7,8 +7,8 @@
 //
 // Both run ffn_kernel on CTA pairs (2-CTA clusters, one CTA per SM).  The WEIGHTS are the M operand of
 // tcgen05.mma cta_group::2 (M = 256 weight rows, 128 per CTA) and the TOKEN rows of the tile are the N
-// operand: N = the tile's rows rounded up to 32, at most 256.  Tensor-core work, shared-memory fill and
-// TMEM columns of a tile therefore follow the rows it really holds - a group of 45 rows costs a 64-column
+// operand: N = the tile's rows rounded up to 16, at most 256.  Tensor-core work, shared-memory fill and
+// TMEM columns of a tile therefore follow the rows it really holds - a group of 45 rows costs a 48-column
 // tile, not a 128- or 256-row one - and a group is cut into ceil(rows / 256) tiles of nearly equal size.
 // Every k-step issues two MMAs that share the token operand:
 //   gate/up: W0 = 256 rows of W_gate, W1 = the same 256 rows of W_up.  The TMEM lane that holds gate
@@ -187,11 +187,16 @@ __device__ __forceinline__ float silu_mul(uint32_t g_bits, uint32_t u_bits) {
   return fmaf(h, t, h) * u;
 }
 
-// Accumulator columns of a tile of `valid_rows` token rows.
+// Accumulator columns of a tile of `valid_rows` token rows: rounded up to 16 (each CTA of the pair supplies half
+// of them, whole 8-row groups of the swizzled layout).
 __device__ __forceinline__ int tile_cols(int valid_rows) {
-  const int n = (valid_rows + 31) & ~31;
+  const int n = (valid_rows + 15) & ~15;
   return n > kTileRows ? kTileRows : n;
 }
+// Columns of a merged tile of n 16-row slots: an even number of slots, so that neither CTA's half cuts a slot.
+__device__ __forceinline__ int merged_cols(int n_slots) { return ((n_slots + 1) & ~1) * kSlotRows; }
+// Columns of a tile from its list entry (y = rows, or minus the slot count of a merged tile).
+__device__ __forceinline__ int entry_cols(int y) { return y < 0 ? merged_cols(-y) : tile_cols(y); }
 
 // ---- the grouped GEMM kernel -----------------------------------------------------------------
 // PHASE 1: gate/up + SwiGLU (256 outputs per tile);  PHASE 2: down (512 outputs per tile).
@@ -201,7 +206,7 @@ template <int PHASE>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_kernel(const __grid_constant__ CUtensorMap tmT128, const __grid_constant__ CUtensorMap tmT64,
            const __grid_constant__ CUtensorMap tmT32, const __grid_constant__ CUtensorMap tmT16,
-           const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
+           const __grid_constant__ CUtensorMap tmT8, const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
            const int4* __restrict__ work, const int2* __restrict__ slots, const int32_t* __restrict__ work_count,
            bf16* __restrict__ out, int ld_out, int n_out, int k_total, int* status) {
   EB_GRID_DEP_SYNC();
@@ -236,6 +241,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmT128, const __grid_constant__ C
     prefetch_tmap(&tmT64);
     prefetch_tmap(&tmT32);
     prefetch_tmap(&tmT16);
+    prefetch_tmap(&tmT8);
     prefetch_tmap(&tmW0);
     prefetch_tmap(&tmW1);
   }
@@ -265,7 +271,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmT128, const __grid_constant__ C
         if (w >= n_work) continue;
         const int4 it = __ldg(work + w);
         const bool merged = it.y < 0;
-        const int half = tile_cols(merged ? -it.y * kSlotRows : it.y) >> 1;   // token rows this CTA loads: a multiple of 16
+        const int half = entry_cols(it.y) >> 1;   // token rows this CTA loads: a multiple of 8 (of 16 in a merged tile)
         const int tok0 = it.x + (int)rank * half;
         // merged tile: this CTA's slots are slots[x + rank * half / 16 ..); a slot beyond the tile's count
         // repeats the first one (its columns are never stored), so the byte count of a stage stays uniform
@@ -293,7 +299,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmT128, const __grid_constant__ C
           } else if (half == 128) {
             tma_pair_load_2d(ta, &tmT128, kb * BK, tok0, fb);
           } else {
-            int r2 = 0;   // rows placed so far; every box starts on a multiple of 16 rows (2 KB), which keeps the swizzle phase
+            int r2 = 0;   // rows placed so far; every box starts on a multiple of 8 rows (1 KB), which keeps the swizzle phase
             if (half & 64) {
               tma_pair_load_2d(ta, &tmT64, kb * BK, tok0, fb);
               r2 = 64;
@@ -302,7 +308,11 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmT128, const __grid_constant__ C
               tma_pair_load_2d(ta + r2 * (BK * 2), &tmT32, kb * BK, tok0 + r2, fb);
               r2 += 32;
             }
-            if (half & 16) tma_pair_load_2d(ta + r2 * (BK * 2), &tmT16, kb * BK, tok0 + r2, fb);
+            if (half & 16) {
+              tma_pair_load_2d(ta + r2 * (BK * 2), &tmT16, kb * BK, tok0 + r2, fb);
+              r2 += 16;
+            }
+            if (half & 8) tma_pair_load_2d(ta + r2 * (BK * 2), &tmT8, kb * BK, tok0 + r2, fb);
           }
           if (++stage == NS) {
             stage = 0;
@@ -322,7 +332,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmT128, const __grid_constant__ C
         if (w >= n_work) continue;
         ++local;
         const int4 it = __ldg(work + w);
-        const uint32_t idesc = kIdescBase | ((uint32_t)(tile_cols(it.y < 0 ? -it.y * kSlotRows : it.y) >> 3) << 17);
+        const uint32_t idesc = kIdescBase | ((uint32_t)(entry_cols(it.y) >> 3) << 17);
         if (!mbar_wait(tempty_bar, (uint32_t)(local & 1) ^ 1u, s_abort, status)) goto done;
         tc_fence_after();
         for (int kb = 0; kb < num_kb; ++kb) {
@@ -446,7 +456,7 @@ __global__ void bounded_wait_probe_kernel(long long limit_cycles, int* status, i
 // A group of `rows` rows is cut into ceil(rows / 256) tiles of nearly equal size, so no tile is a short
 // remainder that would still stream a whole weight tile.
 __device__ __forceinline__ int group_tiles(int rows) { return (rows + kTileRows - 1) / kTileRows; }
-// Columns (token rows rounded up to 32) of the largest tile of a group: its cost class.
+// Columns (token rows rounded up to 16) of the largest tile of a group; its cost class is that count in steps of 32.
 __device__ __forceinline__ int group_cols(int rows) {
   const int t = group_tiles(rows);
   return t ? tile_cols((rows + t - 1) / t) : 0;
@@ -495,7 +505,7 @@ __device__ __forceinline__ bool merged_class(const ModelParams& mp, const int* d
   return mx <= kMergeMaxRows;
 }
 
-// Cost classes of the tiles: class c holds the positions whose tiles have 32 (c + 1) columns.
+// Cost classes of the tiles: class c holds the positions whose tiles have 32 c + 1 .. 32 (c + 1) columns.
 constexpr int kClasses = kTileRows / 32;
 
 // Block-wide exclusive scan (1024 threads) of one value per thread that belongs to one of kClasses classes:
@@ -583,14 +593,14 @@ plan_kernel(ModelParams mp, const int32_t* __restrict__ group_off, const int32_t
         pslots[i] = n_slots;
         if (i == head && n_slots > 0) {   // the class's tiles sit at its first position
           tiles = (n_slots + kMergeSlots - 1) / kMergeSlots;
-          cols = tile_cols(kSlotRows * (n_slots < kMergeSlots ? n_slots : kMergeSlots));
+          cols = merged_cols(n_slots < kMergeSlots ? n_slots : kMergeSlots);
         }
       } else {
         tiles = group_tiles(rows);
         cols = group_cols(rows);
       }
     }
-    const int cls = tiles > 0 ? cols / 32 - 1 : -1;
+    const int cls = tiles > 0 ? (cols + 31) / 32 - 1 : -1;
     long long before[kClasses];
 #pragma unroll
     for (int c = 0; c < kClasses; ++c) before[c] = total[c];
@@ -759,7 +769,7 @@ cudaError_t launch_ffn(eb_ctx* c, cudaStream_t st, const CUtensorMap* tT, const 
   const int2* slots = c->slots;
   const int32_t* wc = c->work_count;
   ++g_ebi_launches;
-  return cudaLaunchKernelEx(&cfg, ffn_kernel<PHASE>, tT[0], tT[1], tT[2], tT[3], tW0, tW1, work, slots, wc, out, ld_out, n_out,
+  return cudaLaunchKernelEx(&cfg, ffn_kernel<PHASE>, tT[0], tT[1], tT[2], tT[3], tT[4], tW0, tW1, work, slots, wc, out, ld_out, n_out,
                             k_total, c->d_status);
 }
 
@@ -814,10 +824,10 @@ eb_status ebi_ffn_run(eb_ctx* c, cudaStream_t st, const void* xp, const int32_t*
   if (!c->ws) return ebi_fail(c, EB_ERR_WORKSPACE, "no workspace set");
   const eb_config& g = c->cfg;
   const int rows = ebi_rows_cap(c);
-  // token-row boxes of 128 / 64 / 32 / 16 rows x one k-block, over the permuted rows and over the intermediate
-  CUtensorMap tok_x[4], tok_a[4];
-  const int box_rows[4] = {128, 64, 32, 16};
-  for (int i = 0; i < 4; ++i)
+  // token-row boxes of 128 / 64 / 32 / 16 / 8 rows x one k-block, over the permuted rows and over the intermediate
+  CUtensorMap tok_x[5], tok_a[5];
+  const int box_rows[5] = {128, 64, 32, 16, 8};
+  for (int i = 0; i < 5; ++i)
     if (!make_map(&tok_x[i], xp, g.H, rows, 0, BK, box_rows[i]) || !make_map(&tok_a[i], c->act, g.I, rows, 0, BK, box_rows[i]))
       return ebi_fail(c, EB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the activations");
   const int nt1 = (g.I + kFeat1 - 1) / kFeat1, nt2 = (g.H + kFeat2 - 1) / kFeat2;

@@ -22,7 +22,7 @@ def _sample_rows(r0, r1):
     """Rows of a group worth comparing at full size: its first and last rows, and the rows around every
     place where the expert kernels change tile or CTA.  Groups of at most 128 rows are one tile of a single
     CTA; larger groups are cut into ceil(rows / 256) nearly equal tiles, each shared by two CTAs that split
-    its rows (rounded up to 32) in halves."""
+    its rows (rounded up to 16) in halves."""
     n = r1 - r0
     if n <= 64:
         return np.arange(r0, r1)
@@ -35,7 +35,7 @@ def _sample_rows(r0, r1):
         start = 0
         for i in range(t):
             rows = each + (1 if i < more else 0)
-            half = ((rows + 31) // 32 * 32) // 2
+            half = ((rows + 15) // 16 * 16) // 2
             for c in (start, start + half, start + rows):
                 pick |= set(range(max(0, c - 8), min(n, c + 8)))
             start += rows
@@ -451,12 +451,12 @@ def test_argument_errors_return_codes():
 # ----------------------------------------------------------------------------------- CTA-pair tiles
 @pytest.mark.parametrize("H,I", [(192, 328), (520, 264)])
 def test_group_sizes_around_the_tile_boundaries(H, I):
-    """Exact group sizes on both sides of every place where the expert kernel's tiling changes: the 32-row
+    """Exact group sizes on both sides of every place where the expert kernel's tiling changes: the 16-row
     steps of a tile's column count, the 128 rows one CTA of a pair loads, and the 256-row limit at which a group
     is cut into two, three, four nearly equal tiles; output widths that end inside the first CTA's half of an
     output tile, inside the second, and just past a whole tile.  Every row of every group is compared."""
-    sizes = [1, 16, 31, 32, 33, 63, 64, 65, 96, 97, 128, 129, 160, 255, 256, 257, 288, 511, 512, 513, 767, 768, 769,
-             1000, 0]
+    sizes = [1, 8, 15, 16, 17, 31, 32, 33, 48, 63, 64, 65, 96, 97, 112, 128, 129, 144, 160, 255, 256, 257, 288, 511, 512,
+             513, 767, 768, 769, 1000, 0]
     E = len(sizes)
     wl = synth.Workload(name="tiles", L=1, E=E, K=1, S=0, H=H, I=I, D=2, mapping="mod", N=1, T=sum(sizes),
                         zipf_s=0.0)
